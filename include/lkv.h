@@ -1,0 +1,249 @@
+/*
+ * lkv.h -- C ABI of the recurrent-layer half of hybrid position-independent
+ * caching ("LinearKV"), hand-written for NVIDIA B200 (sm_100a).
+ *
+ * A hybrid LLM keeps, per recurrent layer and head, a fixed-size state
+ * S in R^{d_k x d_v} that follows the affine recurrence S_i = T_i S_{i-1} + u_i
+ * (Eq. 1).  Serving a request from K independently cached chunks needs two
+ * things from each recurrent layer, and this library provides exactly those:
+ *
+ *   1. lkv_init_state*      S_init = f(S_1 .. S_K)                   (Eq. 4)
+ *        f = one cached state (Section 3.2, "Single-block initialization";
+ *            any block index per Appendix A), or
+ *        f = exact composition sum_j (prod_{m>j} T_{C_m}) S_j        (Eq. 6)
+ *            with scalar transitions for Mamba-2 and dense d_k x d_k
+ *            transitions for Gated DeltaNet (Eq. 5, Eq. 2, Eq. 3);
+ *   2. lkv_gdn_fwd / lkv_ssd_fwd   advance the recurrence from S_init through
+ *        a run of tokens in context order, returning the per-token outputs
+ *        and the final state (Algorithm 1, line 3; Eq. 1-3), computed in the
+ *        chunkwise-parallel form.
+ *
+ * General rules
+ *   - Every data pointer is a DEVICE pointer unless its comment says HOST.
+ *     Small index arrays (chunk ids, cu_k, sel_index, cu_seqlens) are HOST
+ *     int32 arrays: they are range-checked on the host before anything is
+ *     launched and copied to the device by the call itself (into the
+ *     caller's workspace).  They may be reused as soon as the call returns.
+ *   - The caller owns every buffer.  The library allocates nothing, frees
+ *     nothing and keeps no pointer after a call returns; scratch lives in a
+ *     caller-provided workspace whose size lkv_workspace_bytes() reports.
+ *     A workspace must not be shared by calls that can overlap on the GPU.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream).  They do not synchronise.
+ *   - Return value: 0 (LKV_OK) or a negative LKV_ERR_* code.  All argument
+ *     errors are found on the host before any launch; nothing is written in
+ *     that case.  There is no CPU fallback: an unsupported shape returns
+ *     LKV_ERR_UNSUPPORTED.
+ *   - Device-side waits (TMA / tensor-core completion barriers) are bounded.
+ *     A kernel that gives up sets the status word at the start of the
+ *     workspace and returns; lkv_device_status() reads it.
+ *   - Data pointers must be 16-byte aligned (LKV_ERR_ALIGN otherwise).
+ *   - Outputs must not overlap inputs, except that S_T may be the same buffer
+ *     as S0 in the scan calls.
+ *   - States are row-major [.., d_k, d_v] with d_v contiguous, always fp32 on
+ *     output.  All results are deterministic: the same inputs give the same
+ *     bits on every run.
+ */
+#ifndef LKV_H_
+#define LKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LKV_VERSION 100 /* 0.1.0 */
+
+/* status codes */
+#define LKV_OK 0
+#define LKV_ERR_NULL (-1)           /* a required pointer is NULL */
+#define LKV_ERR_DIM (-2)            /* a dimension is negative, zero where it may not be, or inconsistent */
+#define LKV_ERR_MODE (-3)           /* unknown mode / family / dtype / compute value */
+#define LKV_ERR_INDEX (-4)          /* chunk id, selection index or cu_* entry out of range / not monotone */
+#define LKV_ERR_ALIGN (-5)          /* a data pointer is not 16-byte aligned */
+#define LKV_ERR_UNSUPPORTED (-6)    /* valid request, but no kernel for this shape / dtype */
+#define LKV_ERR_WORKSPACE (-7)      /* workspace missing or too small */
+#define LKV_ERR_CUDA (-8)           /* a CUDA runtime call failed (launch, copy, attribute) */
+#define LKV_ERR_DEVICE_TIMEOUT (-9) /* a bounded device-side wait ran out (reported by lkv_device_status) */
+
+/* recurrence family (Eq. 2 vs Eq. 3) */
+#define LKV_FAMILY_MAMBA2 0
+#define LKV_FAMILY_GDN 1
+
+/* element types */
+#define LKV_DTYPE_F32 0
+#define LKV_DTYPE_BF16 1
+
+/* initialiser f of Eq. 4 */
+#define LKV_INIT_LAST 0  /* S_init = S_K, the last matched chunk (the paper's default) */
+#define LKV_INIT_INDEX 1 /* S_init = S_b for a caller-chosen position b (Appendix A) */
+#define LKV_INIT_EXACT 2 /* S_init = exact composition, Eq. 6 */
+
+/* arithmetic used for the dense contractions */
+#define LKV_COMPUTE_AUTO 0   /* tensor cores where a kernel exists for the shape, else fp32 */
+#define LKV_COMPUTE_FP32 1   /* fp32 FMA on CUDA cores everywhere (tight-tolerance / small shapes) */
+#define LKV_COMPUTE_TENSOR 2 /* tensor cores (bf16 operands in the scans, tf32 in GDN composition),
+                                fp32 accumulate; LKV_ERR_UNSUPPORTED if no such kernel fits */
+
+/* `which` of lkv_workspace_bytes */
+#define LKV_WS_INIT 0
+#define LKV_WS_GDN 1
+#define LKV_WS_SSD 2
+
+/*
+ * Descriptor of lkv_init_state / lkv_init_state_batched.
+ *
+ * The cached artefacts live in POOLS indexed by chunk id, so that one cached
+ * chunk can appear at different positions of different requests:
+ *   states       [n_chunks, H, d_k, d_v]   state_dtype (fp32 or bf16)
+ *   transitions  MAMBA2: float [n_chunks, H]            log of the chunk's scalar decay,
+ *                                                      lambda = A_h * sum_t dt_t
+ *                GDN:    float [n_chunks, H, d_k, d_k]  row-major accumulated transition
+ *                                                      T_C = T_{t_L} ... T_{t_1} (Eq. 5)
+ * For Mamba-2, d_k is d_state (N) and d_v is headdim (P).
+ */
+typedef struct lkv_init_desc {
+    int32_t family;           /* LKV_FAMILY_* */
+    int32_t H;                /* heads that own a state (GDN: value heads) */
+    int32_t d_k;
+    int32_t d_v;
+    int32_t n_chunks;         /* pool size */
+    int32_t state_dtype;      /* dtype of the `states` pool; S0 is always fp32 */
+    int32_t sel_index;        /* lkv_init_state, mode INDEX: position b in [0, K) */
+    int32_t compute;          /* LKV_COMPUTE_* (only GDN exact composition looks at it) */
+    const int32_t *chunk_ids; /* lkv_init_state: HOST int32[K] pool ids in context order; NULL = 0..K-1 */
+    void *workspace;          /* device, >= lkv_workspace_bytes(LKV_WS_INIT, desc, n_req, total_K) */
+    size_t workspace_bytes;
+} lkv_init_desc;
+
+/*
+ * Descriptor of lkv_gdn_fwd.  Token tensors are packed over sequences:
+ *   q, k   [T_total, H_k, d_k]   io_dtype        v  [T_total, H_v, d_v]  io_dtype
+ *   g      float [T_total, H_v]  log-decay, alpha = exp(g) <= 1 expected
+ *   beta   float [T_total, H_v]
+ *   S0,S_T float [n_seq, H_v, d_k, d_v]          o  [T_total, H_v, d_v]  io_dtype
+ * Value head h reads q/k head h / (H_v / H_k).
+ */
+typedef struct lkv_gdn_desc {
+    int32_t T_total;
+    int32_t n_seq;
+    const int32_t *cu_seqlens; /* HOST int32[n_seq + 1], cu[0] = 0, cu[n_seq] = T_total; NULL = one sequence */
+    int32_t H_k;
+    int32_t H_v;               /* multiple of H_k */
+    int32_t d_k;
+    int32_t d_v;
+    int32_t io_dtype;          /* dtype of q, k, v and o */
+    int32_t compute;           /* LKV_COMPUTE_* */
+    float scale;               /* read-out scale; 0 selects d_k^(-1/2) */
+    int32_t reserved;
+    void *workspace;
+    size_t workspace_bytes;
+} lkv_gdn_desc;
+
+/*
+ * Descriptor of lkv_ssd_fwd.
+ *   x  [T_total, H, P] io_dtype      dt float [T_total, H] (already activated, > 0)
+ *   A  float [H] (< 0)               B, C [T_total, G, N] io_dtype
+ *   S0,S_T float [n_seq, H, N, P]    y  [T_total, H, P] io_dtype
+ * Head h reads group h / (H / G).
+ */
+typedef struct lkv_ssd_desc {
+    int32_t T_total;
+    int32_t n_seq;
+    const int32_t *cu_seqlens; /* HOST, as in lkv_gdn_desc */
+    int32_t H;
+    int32_t P;                 /* headdim */
+    int32_t N;                 /* d_state */
+    int32_t G;                 /* groups, divides H */
+    int32_t io_dtype;
+    int32_t compute;
+    void *workspace;
+    size_t workspace_bytes;
+} lkv_ssd_desc;
+
+/*
+ * State initialisation for ONE request (Eq. 4; Algorithm 1, line 1).
+ *
+ *   states, transitions  pools as described at lkv_init_desc (device)
+ *   K                    number of matched chunks, >= 0; their pool ids are d->chunk_ids
+ *   mode                 LKV_INIT_LAST | LKV_INIT_INDEX | LKV_INIT_EXACT
+ *   S0                   out, float [H, d_k, d_v] (device)
+ *
+ * LAST / INDEX copy one stored state (widened exactly if the pool is bf16):
+ * with an fp32 pool S0 is bit-identical to the stored state.  `transitions`
+ * is not read and may be NULL.
+ * EXACT evaluates Eq. 6 as the chain S <- S_{c_1}; S <- T_{c_j} S + S_{c_j}
+ * for j = 2..K (Eq. 5 applied in context order); the transition of the first
+ * chunk is never read.  K == 1 returns S_{c_1} untouched in every mode;
+ * K == 0 returns the zero state.
+ * Errors: NULL states/S0/desc (or transitions in EXACT with K >= 2), bad
+ * mode/family/dtype, K < 0, id outside [0, n_chunks), sel_index outside
+ * [0, K), misaligned pointers, unsupported dims, workspace too small.
+ */
+int lkv_init_state(const void *states, const void *transitions, int K, int mode, void *S0,
+                   const lkv_init_desc *d, void *stream);
+
+/*
+ * The same for n_req requests in one launch (batched / ragged serving).
+ *
+ *   chunk_ids  HOST int32[cu_k[n_req]]  pool ids of all requests, concatenated, each in context order
+ *   cu_k       HOST int32[n_req + 1]    request r owns chunk_ids[cu_k[r] .. cu_k[r+1])
+ *   sel_index  HOST int32[n_req]        mode INDEX: position within each request; ignored otherwise (may be NULL)
+ *   S0         out, float [n_req, H, d_k, d_v]
+ * d->chunk_ids and d->sel_index are ignored.
+ */
+int lkv_init_state_batched(const void *states, const void *transitions, const int32_t *chunk_ids,
+                           const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index, void *S0,
+                           const lkv_init_desc *d, void *stream);
+
+/*
+ * Gated DeltaNet scan from an initial state (Eq. 1 with Eq. 3; Algorithm 1, line 3).
+ * For each sequence and value head, in token order:
+ *     S_t = exp(g_t) (I - beta_t k_t k_t^T) S_{t-1} + beta_t k_t v_t^T
+ *     o_t = scale * S_t^T q_t
+ * evaluated chunkwise: inside a block of tokens the triangular system that
+ * couples the tokens (WY / UT transform) is solved at once, and the state is
+ * carried from block to block.  S0 == NULL starts from the empty state;
+ * S_T == NULL skips the final-state write; S_T may alias S0.  Sequences of
+ * any length >= 0 are accepted (no padding is required).
+ */
+int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream);
+
+/*
+ * Mamba-2 (SSD) scan from an initial state (Eq. 1 with Eq. 2; Algorithm 1, line 3).
+ * For each sequence and head, in token order:
+ *     S_t = exp(dt_t A_h) S_{t-1} + dt_t B_t x_t^T,      y_t = S_t^T C_t
+ * evaluated chunkwise (intra-block masked contraction + inter-block state carry).
+ * NULL conventions as in lkv_gdn_fwd.
+ */
+int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
+                const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream);
+
+/*
+ * Workspace size in bytes for a call described by `desc` (lkv_init_desc, lkv_gdn_desc or
+ * lkv_ssd_desc according to `which`).  n_units is the number of requests (init) or
+ * sequences (scans) and n_index the total number of chunk ids over all requests
+ * (init; 0 for the scans).  Returns 0 for a NULL or invalid descriptor.
+ */
+size_t lkv_workspace_bytes(int which, const void *desc, int n_units, int n_index);
+
+/*
+ * Reads the device status word of a workspace: synchronises `stream`, copies 4 bytes to
+ * the host, and returns LKV_OK or LKV_ERR_DEVICE_TIMEOUT (LKV_ERR_CUDA if the copy fails).
+ * The only call here that blocks the host.
+ */
+int lkv_device_status(const void *workspace, void *stream);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char *lkv_status_string(int status);
+
+/* LKV_VERSION of the loaded library. */
+int lkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LKV_H_ */

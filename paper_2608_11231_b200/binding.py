@@ -1,0 +1,243 @@
+"""ctypes binding of the lkv C ABI (see include/lkv.h): argument marshalling only.
+
+Functions carry the names of the C entry points and take torch CUDA tensors for
+device buffers; torch is used for device memory and streams, nothing else.
+Every step of the computation runs in the CUDA library.  There is no fallback:
+if ``liblkv.so`` is missing, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblkv.so")
+
+# constants of include/lkv.h
+LKV_OK = 0
+LKV_ERR_NULL, LKV_ERR_DIM, LKV_ERR_MODE, LKV_ERR_INDEX, LKV_ERR_ALIGN = -1, -2, -3, -4, -5
+LKV_ERR_UNSUPPORTED, LKV_ERR_WORKSPACE, LKV_ERR_CUDA, LKV_ERR_DEVICE_TIMEOUT = -6, -7, -8, -9
+LKV_FAMILY_MAMBA2, LKV_FAMILY_GDN = 0, 1
+LKV_DTYPE_F32, LKV_DTYPE_BF16 = 0, 1
+LKV_INIT_LAST, LKV_INIT_INDEX, LKV_INIT_EXACT = 0, 1, 2
+LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
+LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
+
+EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_gdn_fwd", "lkv_ssd_fwd",
+           "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
+
+
+class lkv_init_desc(ctypes.Structure):
+    _fields_ = [("family", ctypes.c_int32), ("H", ctypes.c_int32), ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32),
+                ("n_chunks", ctypes.c_int32), ("state_dtype", ctypes.c_int32), ("sel_index", ctypes.c_int32),
+                ("compute", ctypes.c_int32), ("chunk_ids", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class lkv_gdn_desc(ctypes.Structure):
+    _fields_ = [("T_total", ctypes.c_int32), ("n_seq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p),
+                ("H_k", ctypes.c_int32), ("H_v", ctypes.c_int32), ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32),
+                ("io_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("scale", ctypes.c_float),
+                ("reserved", ctypes.c_int32), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
+class lkv_ssd_desc(ctypes.Structure):
+    _fields_ = [("T_total", ctypes.c_int32), ("n_seq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p),
+                ("H", ctypes.c_int32), ("P", ctypes.c_int32), ("N", ctypes.c_int32), ("G", ctypes.c_int32),
+                ("io_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class LkvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load liblkv.so (built in-tree by build.py).  Raises if it is missing: there is no fallback path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_11231_b200.build` "
+                               "(or __graft_entry__.build()); the library has no CPU or PyTorch fallback")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        lib.lkv_init_state.argtypes = [vp, vp, ci, ci, vp, ctypes.POINTER(lkv_init_desc), vp]
+        lib.lkv_init_state_batched.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, ctypes.POINTER(lkv_init_desc), vp]
+        lib.lkv_gdn_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), vp]
+        lib.lkv_ssd_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_ssd_desc), vp]
+        lib.lkv_workspace_bytes.argtypes = [ci, vp, ci, ci]
+        lib.lkv_workspace_bytes.restype = ctypes.c_size_t
+        lib.lkv_device_status.argtypes = [vp, vp]
+        lib.lkv_status_string.argtypes = [ci]
+        lib.lkv_status_string.restype = ctypes.c_char_p
+        for name in ("lkv_init_state", "lkv_init_state_batched", "lkv_gdn_fwd", "lkv_ssd_fwd",
+                     "lkv_device_status", "lkv_version"):
+            getattr(lib, name).restype = ci
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().lkv_status_string(int(status)).decode()
+
+
+def lkv_version() -> int:
+    return int(load().lkv_version())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LKV_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return LKV_DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("device buffers must be contiguous CUDA tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _host_i32(a) -> Optional[np.ndarray]:
+    if a is None:
+        return None
+    if isinstance(a, torch.Tensor):
+        a = a.cpu().numpy()
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _hp(a: Optional[np.ndarray]):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+_ws_cache = {}
+
+
+def workspace(device, nbytes: int) -> torch.Tensor:
+    """A zero-initialised, cached device workspace of at least nbytes (one per device and stream)."""
+    key = (torch.device(device).index, torch.cuda.current_stream().cuda_stream)
+    ws = _ws_cache.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.zeros(max(int(nbytes), 4096), dtype=torch.uint8, device=device)
+        _ws_cache[key] = ws
+    return ws
+
+
+def lkv_workspace_bytes(which: int, desc, n_units: int, n_index: int = 0) -> int:
+    return int(load().lkv_workspace_bytes(which, ctypes.cast(ctypes.pointer(desc), ctypes.c_void_p), n_units, n_index))
+
+
+def lkv_device_status(ws: torch.Tensor, stream=None) -> int:
+    return int(load().lkv_device_status(_ptr(ws), _stream(stream)))
+
+
+def _init_desc(states, family, compute, ws_t, n_units, n_index, chunk_ids_np=None, sel_index=0):
+    n, H, d_k, d_v = states.shape
+    d = lkv_init_desc(family=family, H=H, d_k=d_k, d_v=d_v, n_chunks=n, state_dtype=_dtype_code(states),
+                      sel_index=int(sel_index), compute=compute,
+                      chunk_ids=None if chunk_ids_np is None else chunk_ids_np.ctypes.data, workspace=None,
+                      workspace_bytes=0)
+    if ws_t is None:
+        ws_t = workspace(states.device, lkv_workspace_bytes(LKV_WS_INIT, d, n_units, n_index))
+    d.workspace = ws_t.data_ptr()
+    d.workspace_bytes = ws_t.numel()
+    return d, ws_t
+
+
+def lkv_init_state(states: torch.Tensor, transitions: Optional[torch.Tensor], K: int, mode: int,
+                   S0: Optional[torch.Tensor] = None, *, family: int, chunk_ids=None, sel_index: int = 0,
+                   compute: int = LKV_COMPUTE_AUTO, workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """State initialisation for one request.  states: pool [n, H, d_k, d_v]; returns S0 [H, d_k, d_v] fp32."""
+    ids = _host_i32(chunk_ids)
+    d, ws_t = _init_desc(states, family, compute, workspace_t, 1, int(K), ids, sel_index)
+    if S0 is None:
+        S0 = torch.empty(states.shape[1:], dtype=torch.float32, device=states.device)
+    st = load().lkv_init_state(_ptr(states), _ptr(transitions), int(K), int(mode), _ptr(S0), ctypes.byref(d),
+                               _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_init_state")
+    return S0
+
+
+def lkv_init_state_batched(states: torch.Tensor, transitions: Optional[torch.Tensor], chunk_ids, cu_k, n_req: int,
+                           mode: int, sel_index=None, S0: Optional[torch.Tensor] = None, *, family: int,
+                           compute: int = LKV_COMPUTE_AUTO, workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """State initialisation for n_req requests in one launch; returns S0 [n_req, H, d_k, d_v] fp32."""
+    ids, cu, sel = _host_i32(chunk_ids), _host_i32(cu_k), _host_i32(sel_index)
+    d, ws_t = _init_desc(states, family, compute, workspace_t, int(n_req), 0 if ids is None else ids.size)
+    if S0 is None:
+        S0 = torch.empty((n_req,) + tuple(states.shape[1:]), dtype=torch.float32, device=states.device)
+    st = load().lkv_init_state_batched(_ptr(states), _ptr(transitions), _hp(ids), _hp(cu), int(n_req), int(mode),
+                                       _hp(sel), _ptr(S0), ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_init_state_batched")
+    return S0
+
+
+def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None, scale: float = 0.0,
+                compute: int = LKV_COMPUTE_AUTO, want_final_state: bool = True,
+                workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """Gated DeltaNet scan.  q, k: [T, H_k, d_k]; v: [T, H_v, d_v]; g, beta: [T, H_v] fp32.
+
+    Returns (o [T, H_v, d_v] in the dtype of v, S_T [n_seq, H_v, d_k, d_v] fp32 or None).
+    """
+    T, H_k, d_k = q.shape
+    _, H_v, d_v = v.shape
+    cu = _host_i32(cu_seqlens)
+    n_seq = 1 if cu is None else cu.size - 1
+    d = lkv_gdn_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H_k=H_k, H_v=H_v,
+                     d_k=d_k, d_v=d_v, io_dtype=_dtype_code(v), compute=compute, scale=float(scale), reserved=0,
+                     workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(v.device, lkv_workspace_bytes(LKV_WS_GDN, d, n_seq))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    if o is None:
+        o = torch.empty_like(v)
+    if S_T is None and want_final_state:
+        S_T = torch.empty((n_seq, H_v, d_k, d_v), dtype=torch.float32, device=v.device)
+    st = load().lkv_gdn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S0), _ptr(o), _ptr(S_T),
+                            ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_gdn_fwd")
+    return o, S_T
+
+
+def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, compute: int = LKV_COMPUTE_AUTO,
+                want_final_state: bool = True, workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """Mamba-2 (SSD) scan.  x: [T, H, P]; dt: [T, H] fp32; A: [H] fp32; B, C: [T, G, N].
+
+    Returns (y [T, H, P] in the dtype of x, S_T [n_seq, H, N, P] fp32 or None).
+    """
+    T, H, P = x.shape
+    _, G, N = B.shape
+    cu = _host_i32(cu_seqlens)
+    n_seq = 1 if cu is None else cu.size - 1
+    d = lkv_ssd_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H=H, P=P, N=N, G=G,
+                     io_dtype=_dtype_code(x), compute=compute, workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(x.device, lkv_workspace_bytes(LKV_WS_SSD, d, n_seq))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    if y is None:
+        y = torch.empty_like(x)
+    if S_T is None and want_final_state:
+        S_T = torch.empty((n_seq, H, N, P), dtype=torch.float32, device=x.device)
+    st = load().lkv_ssd_fwd(_ptr(x), _ptr(dt), _ptr(A), _ptr(B), _ptr(C), _ptr(S0), _ptr(y), _ptr(S_T),
+                            ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_ssd_fwd")
+    return y, S_T

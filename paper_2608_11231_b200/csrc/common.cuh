@@ -1,0 +1,99 @@
+// Shared device/host helpers of the lkv CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lkv.h"
+
+namespace lkv {
+
+// First 256 bytes of every workspace: word 0 is the device status (0 = fine).
+constexpr size_t kWsHeaderBytes = 256;
+// Status values written by kernels whose bounded waits ran out.
+constexpr int kDevTimeout = 1;
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+template <typename T>
+__device__ __forceinline__ float to_f32(T x);
+template <>
+__device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T>
+__device__ __forceinline__ T from_f32(float x);
+template <>
+__device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Small host-checked index arrays travel to the device inside the kernel parameters
+// (no copy, no extra stream operation); lists longer than CAP are copied into the
+// caller's workspace instead and reached through `ptr`.
+template <int CAP>
+struct IndexBlock {
+    const int32_t *ptr;  // device copy, or nullptr when the inline array is used
+    int32_t v[CAP];
+    __device__ __forceinline__ int32_t operator[](int i) const { return ptr ? ptr[i] : v[i]; }
+};
+constexpr int kInitIdxCap = 4000;  // ints: cu_k | sel | ids
+constexpr int kScanIdxCap = 1000;  // ints: cu_seqlens
+
+// Launch-side records shared by the entry points and the kernels.  Passed by value as
+// __grid_constant__ kernel parameters.
+struct InitArgs {
+    const void *states;        // pool
+    const float *transitions;  // pool (log-decay or dense)
+    float *S0;                 // [n_req, H, d_k, d_v]
+    int32_t n_req, H, d_k, d_v;
+    int32_t off_sel;           // offset of sel[n_req] in idx, or -1 (= last block)
+    int32_t off_ids;           // offset of ids[total_K] in idx; cu_k[n_req + 1] sits at 0
+    int32_t *status;           // device status word
+    IndexBlock<kInitIdxCap> idx;
+    __device__ __forceinline__ int cu_k(int r) const { return idx[r]; }
+    __device__ __forceinline__ int id(int i) const { return idx[off_ids + i]; }
+    __device__ __forceinline__ int sel(int r, int K) const { return off_sel < 0 ? K - 1 : idx[off_sel + r]; }
+};
+
+struct GdnArgs {
+    const void *q, *k, *v;
+    const float *g, *beta, *S0;
+    void *o;
+    float *S_T;
+    int32_t n_seq, H_k, H_v, d_k, d_v;
+    float scale;
+    int32_t *status;
+    IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
+};
+
+struct SsdArgs {
+    const void *x, *B, *C;
+    const float *dt, *A, *S0;
+    void *y;
+    float *S_T;
+    int32_t n_seq, H, P, N, G;
+    int32_t *status;
+    IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
+};
+
+// Kernel launchers (one translation unit each); all return a cudaError_t from the launch.
+cudaError_t launch_init_single(const InitArgs &a, bool pool_bf16, cudaStream_t s);
+cudaError_t launch_init_mamba_exact(const InitArgs &a, bool pool_bf16, cudaStream_t s);
+cudaError_t launch_init_gdn_exact_fp32(const InitArgs &a, bool pool_bf16, cudaStream_t s);
+bool init_gdn_exact_tensor_supported(const InitArgs &a, bool pool_bf16);
+cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, cudaStream_t s);
+
+bool gdn_scan_fp32_supported(int d_k, int d_v);
+cudaError_t launch_gdn_scan_fp32(const GdnArgs &a, bool io_bf16, cudaStream_t s);
+bool gdn_scan_tensor_supported(const GdnArgs &a, bool io_bf16);
+cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s);
+
+bool ssd_scan_fp32_supported(int N, int P);
+cudaError_t launch_ssd_scan_fp32(const SsdArgs &a, bool io_bf16, cudaStream_t s);
+bool ssd_scan_tensor_supported(const SsdArgs &a, bool io_bf16);
+cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s);
+
+}  // namespace lkv

@@ -1,0 +1,296 @@
+// C-ABI entry points: argument validation, index marshalling and kernel selection.
+// Everything that can be wrong with a call is found here, on the host, before a launch.
+#include <string.h>
+
+#include <vector>
+
+#include "common.cuh"
+
+using namespace lkv;
+
+namespace {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool dtype_ok(int d) { return d == LKV_DTYPE_F32 || d == LKV_DTYPE_BF16; }
+inline bool compute_ok(int c) { return c == LKV_COMPUTE_AUTO || c == LKV_COMPUTE_FP32 || c == LKV_COMPUTE_TENSOR; }
+
+size_t ws_bytes_for(int n_ints, int cap) {
+    return kWsHeaderBytes + (n_ints > cap ? align_up(sizeof(int32_t) * static_cast<size_t>(n_ints), 256) : 0);
+}
+
+// Puts `ints` where the kernels will find them: inline in the parameter block when they
+// fit, otherwise one small async copy into the workspace behind its header.
+template <int CAP>
+int place_indices(IndexBlock<CAP> &blk, const std::vector<int32_t> &ints, void *workspace, cudaStream_t s) {
+    if (static_cast<int>(ints.size()) <= CAP) {
+        blk.ptr = nullptr;
+        if (!ints.empty()) memcpy(blk.v, ints.data(), sizeof(int32_t) * ints.size());
+        return LKV_OK;
+    }
+    int32_t *dst = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + kWsHeaderBytes);
+    if (cudaMemcpyAsync(dst, ints.data(), sizeof(int32_t) * ints.size(), cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    blk.ptr = dst;
+    return LKV_OK;
+}
+
+int check_init_desc(const lkv_init_desc *d) {
+    if (!d) return LKV_ERR_NULL;
+    if (d->family != LKV_FAMILY_MAMBA2 && d->family != LKV_FAMILY_GDN) return LKV_ERR_MODE;
+    if (!dtype_ok(d->state_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
+    if (d->H < 1 || d->d_k < 1 || d->d_v < 1 || d->n_chunks < 0) return LKV_ERR_DIM;
+    return LKV_OK;
+}
+
+int init_impl(const void *states, const void *transitions, const int32_t *chunk_ids, const int32_t *cu_k,
+              int n_req, int mode, const int32_t *sel_index, void *S0, const lkv_init_desc *d, void *stream) {
+    int st = check_init_desc(d);
+    if (st != LKV_OK) return st;
+    if (mode != LKV_INIT_LAST && mode != LKV_INIT_INDEX && mode != LKV_INIT_EXACT) return LKV_ERR_MODE;
+    if (n_req < 0) return LKV_ERR_DIM;
+    if (!cu_k) return LKV_ERR_NULL;
+    if (cu_k[0] != 0) return LKV_ERR_INDEX;
+    int max_k = 0;
+    for (int r = 0; r < n_req; ++r) {
+        if (cu_k[r + 1] < cu_k[r]) return LKV_ERR_INDEX;
+        max_k = cu_k[r + 1] - cu_k[r] > max_k ? cu_k[r + 1] - cu_k[r] : max_k;
+    }
+    const int total = cu_k[n_req];
+    if (total > 0 && !chunk_ids) return LKV_ERR_NULL;
+    for (int i = 0; i < total; ++i)
+        if (chunk_ids[i] < 0 || chunk_ids[i] >= d->n_chunks) return LKV_ERR_INDEX;
+    if (mode == LKV_INIT_INDEX) {
+        if (n_req > 0 && !sel_index) return LKV_ERR_NULL;
+        for (int r = 0; r < n_req; ++r) {
+            const int K = cu_k[r + 1] - cu_k[r];
+            if (K > 0 && (sel_index[r] < 0 || sel_index[r] >= K)) return LKV_ERR_INDEX;
+        }
+    }
+    if (n_req == 0) return LKV_OK;
+    if (!S0) return LKV_ERR_NULL;
+    if (total > 0 && !states) return LKV_ERR_NULL;
+    const bool exact = mode == LKV_INIT_EXACT && max_k >= 2;
+    if (exact && !transitions) return LKV_ERR_NULL;
+    if (!aligned16(S0) || !aligned16(states) || (exact && !aligned16(transitions))) return LKV_ERR_ALIGN;
+    const bool pool_bf16 = d->state_dtype == LKV_DTYPE_BF16;
+    if (d->d_v % (pool_bf16 ? 8 : 4) != 0) return LKV_ERR_UNSUPPORTED;
+
+    const int n_ints = (n_req + 1) + (mode == LKV_INIT_INDEX ? n_req : 0) + total;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(n_ints, kInitIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+
+    InitArgs a;
+    a.states = states;
+    a.transitions = static_cast<const float *>(transitions);
+    a.S0 = static_cast<float *>(S0);
+    a.n_req = n_req;
+    a.H = d->H;
+    a.d_k = d->d_k;
+    a.d_v = d->d_v;
+    a.status = static_cast<int32_t *>(d->workspace);
+    std::vector<int32_t> ints;
+    ints.reserve(n_ints);
+    ints.insert(ints.end(), cu_k, cu_k + n_req + 1);
+    a.off_sel = -1;
+    if (mode == LKV_INIT_INDEX) {
+        a.off_sel = static_cast<int32_t>(ints.size());
+        ints.insert(ints.end(), sel_index, sel_index + n_req);
+    }
+    a.off_ids = static_cast<int32_t>(ints.size());
+    if (total > 0) ints.insert(ints.end(), chunk_ids, chunk_ids + total);
+
+    // kernel choice (no launch has happened yet: an unsupported request leaves everything untouched)
+    enum { kSingle, kMamba, kGdnFp32, kGdnTensor } which;
+    if (!exact) {
+        which = kSingle;  // LAST, INDEX, and EXACT with K <= 1 everywhere are plain copies
+        a.off_sel = (mode == LKV_INIT_INDEX) ? a.off_sel : -1;
+    } else if (d->family == LKV_FAMILY_MAMBA2) {
+        which = kMamba;
+    } else {
+        const bool tensor_fits = init_gdn_exact_tensor_supported(a, pool_bf16);
+        if (d->compute == LKV_COMPUTE_TENSOR && !tensor_fits) return LKV_ERR_UNSUPPORTED;
+        which = (d->compute != LKV_COMPUTE_FP32 && tensor_fits) ? kGdnTensor : kGdnFp32;
+        if (which == kGdnFp32 && (2 * d->d_k * 32 + 32 * (d->d_k + 1)) * sizeof(float) > 227 * 1024) return LKV_ERR_UNSUPPORTED;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = place_indices(a.idx, ints, d->workspace, s);
+    if (st != LKV_OK) return st;
+    cudaError_t e = cudaSuccess;
+    switch (which) {
+        case kSingle: e = launch_init_single(a, pool_bf16, s); break;
+        case kMamba: e = launch_init_mamba_exact(a, pool_bf16, s); break;
+        case kGdnFp32: e = launch_init_gdn_exact_fp32(a, pool_bf16, s); break;
+        case kGdnTensor: e = launch_init_gdn_exact_tensor(a, s); break;
+    }
+    return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
+// Shared checks of the two scan descriptors' sequence layout; fills `cu` with the
+// offsets the kernels will use.
+int check_seqs(int T_total, int n_seq, const int32_t *cu_seqlens, std::vector<int32_t> &cu) {
+    if (T_total < 0 || n_seq < 0) return LKV_ERR_DIM;
+    if (!cu_seqlens) {
+        if (n_seq != 1) return LKV_ERR_NULL;
+        cu = {0, T_total};
+        return LKV_OK;
+    }
+    if (cu_seqlens[0] != 0 || cu_seqlens[n_seq] != T_total) return LKV_ERR_INDEX;
+    for (int i = 0; i < n_seq; ++i)
+        if (cu_seqlens[i + 1] < cu_seqlens[i]) return LKV_ERR_INDEX;
+    cu.assign(cu_seqlens, cu_seqlens + n_seq + 1);
+    return LKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lkv_init_state(const void *states, const void *transitions, int K, int mode, void *S0,
+                   const lkv_init_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (K < 0) return LKV_ERR_DIM;
+    std::vector<int32_t> ids;
+    const int32_t *idp = d->chunk_ids;
+    if (!idp) {
+        ids.resize(K);
+        for (int i = 0; i < K; ++i) ids[i] = i;
+        idp = ids.data();
+    }
+    const int32_t cu_k[2] = {0, K};
+    const int32_t sel[1] = {d->sel_index};
+    return init_impl(states, transitions, idp, cu_k, 1, mode, sel, S0, d, stream);
+}
+
+int lkv_init_state_batched(const void *states, const void *transitions, const int32_t *chunk_ids,
+                           const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index, void *S0,
+                           const lkv_init_desc *d, void *stream) {
+    return init_impl(states, transitions, chunk_ids, cu_k, n_req, mode, sel_index, S0, d, stream);
+}
+
+int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
+    if (d->H_k < 1 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1 || d->H_v % d->H_k != 0) return LKV_ERR_DIM;
+    std::vector<int32_t> cu;
+    int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
+    if (st != LKV_OK) return st;
+    if (d->n_seq == 0) return LKV_OK;
+    if (d->T_total > 0 && (!q || !k || !v || !g || !beta || !o)) return LKV_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(S0) ||
+        !aligned16(o) || !aligned16(S_T))
+        return LKV_ERR_ALIGN;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+
+    GdnArgs a;
+    a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = S_T;
+    a.n_seq = d->n_seq; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
+    a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
+    a.status = static_cast<int32_t *>(d->workspace);
+    const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
+    const bool tensor_fits = gdn_scan_tensor_supported(a, io_bf16);
+    const bool fp32_fits = gdn_scan_fp32_supported(d->d_k, d->d_v);
+    bool use_tensor;
+    if (d->compute == LKV_COMPUTE_TENSOR) {
+        if (!tensor_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = true;
+    } else if (d->compute == LKV_COMPUTE_FP32) {
+        if (!fp32_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = false;
+    } else {
+        if (!tensor_fits && !fp32_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = tensor_fits;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = place_indices(a.cu, cu, d->workspace, s);
+    if (st != LKV_OK) return st;
+    const cudaError_t e = use_tensor ? launch_gdn_scan_tensor(a, s) : launch_gdn_scan_fp32(a, io_bf16, s);
+    return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
+int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
+                const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
+    if (d->H < 1 || d->P < 1 || d->N < 1 || d->G < 1 || d->H % d->G != 0) return LKV_ERR_DIM;
+    std::vector<int32_t> cu;
+    int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
+    if (st != LKV_OK) return st;
+    if (d->n_seq == 0) return LKV_OK;
+    if (!A) return LKV_ERR_NULL;
+    if (d->T_total > 0 && (!x || !dt || !B || !C || !y)) return LKV_ERR_NULL;
+    if (!aligned16(x) || !aligned16(dt) || !aligned16(A) || !aligned16(B) || !aligned16(C) || !aligned16(S0) ||
+        !aligned16(y) || !aligned16(S_T))
+        return LKV_ERR_ALIGN;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+
+    SsdArgs a;
+    a.x = x; a.dt = dt; a.A = A; a.B = B; a.C = C; a.S0 = S0; a.y = y; a.S_T = S_T;
+    a.n_seq = d->n_seq; a.H = d->H; a.P = d->P; a.N = d->N; a.G = d->G;
+    a.status = static_cast<int32_t *>(d->workspace);
+    const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
+    const bool tensor_fits = ssd_scan_tensor_supported(a, io_bf16);
+    const bool fp32_fits = ssd_scan_fp32_supported(d->N, d->P);
+    bool use_tensor;
+    if (d->compute == LKV_COMPUTE_TENSOR) {
+        if (!tensor_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = true;
+    } else if (d->compute == LKV_COMPUTE_FP32) {
+        if (!fp32_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = false;
+    } else {
+        if (!tensor_fits && !fp32_fits) return LKV_ERR_UNSUPPORTED;
+        use_tensor = tensor_fits;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = place_indices(a.cu, cu, d->workspace, s);
+    if (st != LKV_OK) return st;
+    const cudaError_t e = use_tensor ? launch_ssd_scan_tensor(a, s) : launch_ssd_scan_fp32(a, io_bf16, s);
+    return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
+size_t lkv_workspace_bytes(int which, const void *desc, int n_units, int n_index) {
+    if (!desc || n_units < 0 || n_index < 0) return 0;
+    switch (which) {
+        case LKV_WS_INIT: return ws_bytes_for(2 * n_units + 1 + n_index, kInitIdxCap);
+        case LKV_WS_GDN:
+        case LKV_WS_SSD: return ws_bytes_for(n_units + 1, kScanIdxCap);
+        default: return 0;
+    }
+}
+
+int lkv_device_status(const void *workspace, void *stream) {
+    if (!workspace) return LKV_ERR_NULL;
+    int32_t word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    return word == 0 ? LKV_OK : LKV_ERR_DEVICE_TIMEOUT;
+}
+
+const char *lkv_status_string(int status) {
+    switch (status) {
+        case LKV_OK: return "ok";
+        case LKV_ERR_NULL: return "a required pointer is NULL";
+        case LKV_ERR_DIM: return "bad dimension";
+        case LKV_ERR_MODE: return "unknown mode, family, dtype or compute value";
+        case LKV_ERR_INDEX: return "index out of range or offsets not monotone";
+        case LKV_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case LKV_ERR_UNSUPPORTED: return "no kernel for this shape or dtype";
+        case LKV_ERR_WORKSPACE: return "workspace missing or too small";
+        case LKV_ERR_CUDA: return "CUDA runtime call failed";
+        case LKV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int lkv_version(void) { return LKV_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,159 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol
+the header declares, and rejects bad arguments before anything could be launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2608_11231_b200 import binding as b
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+FAKE = 0x7F0000000000  # a 16-byte aligned non-NULL "device pointer"; never dereferenced on the host
+
+
+@pytest.fixture(scope="module")
+def lib():
+    if not os.path.exists(b.LIB_PATH):
+        import __graft_entry__
+        __graft_entry__.build()
+    return b.load()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    text = open(os.path.join(ROOT, "include", "lkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(lkv_[a-z_0-9]+)\s*\(", text))
+    assert declared == set(b.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert b.lkv_version() == 100
+    seen = {b.status_string(s) for s in range(0, -10, -1)}
+    assert len(seen) == 10 and "unknown status" not in seen
+    assert b.status_string(-99) == "unknown status"
+
+
+def _desc(**kw):
+    base = dict(family=b.LKV_FAMILY_GDN, H=2, d_k=64, d_v=64, n_chunks=4, state_dtype=b.LKV_DTYPE_F32, sel_index=0,
+                compute=b.LKV_COMPUTE_AUTO, chunk_ids=None, workspace=FAKE, workspace_bytes=1 << 20)
+    base.update(kw)
+    return b.lkv_init_desc(**base)
+
+
+def _init(lib, d, K=4, mode=b.LKV_INIT_EXACT, states=FAKE, trans=FAKE, S0=FAKE):
+    return lib.lkv_init_state(states, trans, K, mode, S0, ctypes.byref(d) if d is not None else None, None)
+
+
+def test_init_state_argument_errors(lib):
+    assert _init(lib, None) == b.LKV_ERR_NULL
+    assert _init(lib, _desc(), K=-1) == b.LKV_ERR_DIM
+    assert _init(lib, _desc(), mode=7) == b.LKV_ERR_MODE
+    assert _init(lib, _desc(family=5)) == b.LKV_ERR_MODE
+    assert _init(lib, _desc(state_dtype=9)) == b.LKV_ERR_MODE
+    assert _init(lib, _desc(compute=3)) == b.LKV_ERR_MODE
+    assert _init(lib, _desc(H=0)) == b.LKV_ERR_DIM
+    assert _init(lib, _desc(), K=5) == b.LKV_ERR_INDEX            # implicit ids 0..4 exceed the pool of 4
+    ids = np.array([0, 1, 4, 2], dtype=np.int32)
+    assert _init(lib, _desc(chunk_ids=ids.ctypes.data)) == b.LKV_ERR_INDEX
+    ids = np.array([0, -1, 3, 2], dtype=np.int32)
+    assert _init(lib, _desc(chunk_ids=ids.ctypes.data)) == b.LKV_ERR_INDEX
+    assert _init(lib, _desc(sel_index=4), mode=b.LKV_INIT_INDEX) == b.LKV_ERR_INDEX
+    assert _init(lib, _desc(sel_index=-1), mode=b.LKV_INIT_INDEX) == b.LKV_ERR_INDEX
+    assert _init(lib, _desc(), S0=None) == b.LKV_ERR_NULL
+    assert _init(lib, _desc(), states=None) == b.LKV_ERR_NULL
+    assert _init(lib, _desc(), trans=None) == b.LKV_ERR_NULL      # exact mode with K >= 2 needs transitions
+    assert _init(lib, _desc(), S0=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert _init(lib, _desc(), states=FAKE + 8) == b.LKV_ERR_ALIGN
+    assert _init(lib, _desc(d_v=6)) == b.LKV_ERR_UNSUPPORTED
+    assert _init(lib, _desc(workspace=None)) == b.LKV_ERR_WORKSPACE
+    assert _init(lib, _desc(workspace_bytes=16)) == b.LKV_ERR_WORKSPACE
+    assert _init(lib, _desc(compute=b.LKV_COMPUTE_TENSOR, d_k=24, d_v=24)) == b.LKV_ERR_UNSUPPORTED
+
+
+def test_init_state_batched_argument_errors(lib):
+    d = _desc()
+    ids = np.array([0, 1, 2, 3, 1], dtype=np.int32)
+    f = lib.lkv_init_state_batched
+    call = lambda cu, n, mode=b.LKV_INIT_EXACT, sel=None, idp=ids: f(
+        FAKE, FAKE, idp.ctypes.data if idp is not None else None, cu.ctypes.data if cu is not None else None, n, mode,
+        sel.ctypes.data if sel is not None else None, FAKE, ctypes.byref(d), None)
+    assert call(None, 2) == b.LKV_ERR_NULL
+    assert call(np.array([1, 3, 5], dtype=np.int32), 2) == b.LKV_ERR_INDEX      # must start at 0
+    assert call(np.array([0, 4, 3], dtype=np.int32), 2) == b.LKV_ERR_INDEX      # not monotone
+    assert call(np.array([0, 3, 5], dtype=np.int32), -1) == b.LKV_ERR_DIM
+    assert call(np.array([0, 3, 5], dtype=np.int32), 2, idp=None) == b.LKV_ERR_NULL
+    assert call(np.array([0, 3, 5], dtype=np.int32), 2, mode=b.LKV_INIT_INDEX) == b.LKV_ERR_NULL
+    assert call(np.array([0, 3, 5], dtype=np.int32), 2, mode=b.LKV_INIT_INDEX,
+                sel=np.array([2, 2], dtype=np.int32)) == b.LKV_ERR_INDEX
+    assert call(np.array([0], dtype=np.int32), 0) == b.LKV_OK                    # no requests: nothing to do
+
+
+def _gdn_desc(**kw):
+    base = dict(T_total=100, n_seq=1, cu_seqlens=None, H_k=2, H_v=4, d_k=64, d_v=64, io_dtype=b.LKV_DTYPE_F32,
+                compute=b.LKV_COMPUTE_AUTO, scale=0.0, reserved=0, workspace=FAKE, workspace_bytes=1 << 20)
+    base.update(kw)
+    return b.lkv_gdn_desc(**base)
+
+
+def test_gdn_fwd_argument_errors(lib):
+    f = lambda d, q=FAKE, o=FAKE, S0=None: lib.lkv_gdn_fwd(q, FAKE, FAKE, FAKE, FAKE, S0, o, None,
+                                                           ctypes.byref(d) if d is not None else None, None)
+    assert f(None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(io_dtype=4)) == b.LKV_ERR_MODE
+    assert f(_gdn_desc(H_v=3)) == b.LKV_ERR_DIM
+    assert f(_gdn_desc(d_k=0)) == b.LKV_ERR_DIM
+    assert f(_gdn_desc(T_total=-1)) == b.LKV_ERR_DIM
+    assert f(_gdn_desc(n_seq=2)) == b.LKV_ERR_NULL                      # several sequences need cu_seqlens
+    cu = np.array([0, 60, 90], dtype=np.int32)
+    assert f(_gdn_desc(n_seq=2, cu_seqlens=cu.ctypes.data)) == b.LKV_ERR_INDEX   # does not end at T_total
+    cu = np.array([0, 120, 100], dtype=np.int32)
+    assert f(_gdn_desc(n_seq=2, cu_seqlens=cu.ctypes.data)) == b.LKV_ERR_INDEX
+    assert f(_gdn_desc(), q=None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(), o=FAKE + 2) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(), S0=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(d_v=48)) == b.LKV_ERR_UNSUPPORTED
+    assert f(_gdn_desc(workspace=None)) == b.LKV_ERR_WORKSPACE
+    assert f(_gdn_desc(compute=b.LKV_COMPUTE_TENSOR, d_k=24, d_v=32)) == b.LKV_ERR_UNSUPPORTED
+    assert f(_gdn_desc(n_seq=0, T_total=0, cu_seqlens=np.array([0], dtype=np.int32).ctypes.data)) == b.LKV_OK
+
+
+def _ssd_desc(**kw):
+    base = dict(T_total=100, n_seq=1, cu_seqlens=None, H=8, P=64, N=128, G=2, io_dtype=b.LKV_DTYPE_BF16,
+                compute=b.LKV_COMPUTE_AUTO, workspace=FAKE, workspace_bytes=1 << 20)
+    base.update(kw)
+    return b.lkv_ssd_desc(**base)
+
+
+def test_ssd_fwd_argument_errors(lib):
+    f = lambda d, x=FAKE, A=FAKE, y=FAKE: lib.lkv_ssd_fwd(x, FAKE, A, FAKE, FAKE, None, y, None,
+                                                          ctypes.byref(d) if d is not None else None, None)
+    assert f(None) == b.LKV_ERR_NULL
+    assert f(_ssd_desc(compute=-1)) == b.LKV_ERR_MODE
+    assert f(_ssd_desc(G=3)) == b.LKV_ERR_DIM
+    assert f(_ssd_desc(N=0)) == b.LKV_ERR_DIM
+    assert f(_ssd_desc(), A=None) == b.LKV_ERR_NULL
+    assert f(_ssd_desc(), x=None) == b.LKV_ERR_NULL
+    assert f(_ssd_desc(), y=FAKE + 8) == b.LKV_ERR_ALIGN
+    assert f(_ssd_desc(P=48)) == b.LKV_ERR_UNSUPPORTED
+    assert f(_ssd_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE
+
+
+def test_workspace_bytes(lib):
+    d = _desc()
+    small = b.lkv_workspace_bytes(b.LKV_WS_INIT, d, 1, 8)
+    big = b.lkv_workspace_bytes(b.LKV_WS_INIT, d, 64, 64 * 64)
+    assert small >= 256 and big >= 256 + 4 * (64 * 64 + 129)
+    assert b.lkv_workspace_bytes(b.LKV_WS_GDN, _gdn_desc(), 64) >= 256
+    assert lib.lkv_workspace_bytes(b.LKV_WS_INIT, None, 1, 1) == 0
+    assert b.lkv_workspace_bytes(17, d, 1, 1) == 0
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    monkeypatch.setattr(b, "_lib", None)
+    monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "liblkv.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        b.load()
