@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the recurrent-layer hot path on synthetic data shaped like the paper's workloads.
+
+One "step" is one pass of the whole hot path over one batch: for every recurrent-layer request of the
+workload, single-state initialisation, exact composition, and the chunkwise scan of the request's
+recompute segment from the composed state (both families when the workload has both).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg3|cfg4] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` = context tokens served per second by the step (all requests'
+context tokens / step time), device-timed with inputs resident in HBM; `e2e` = the same with every
+input copied host->device from pinned memory and every result copied back inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_11231_b200 import workloads as wl  # noqa: E402
+
+METRIC = "effective_prefill_tokens_per_s"
+UNIT = "tokens/s"
+GDN_SHAPE = dict(H_k=16, H_v=32, d_k=128, d_v=128)
+SSD_SHAPE = dict(H=80, P=64, N=128, G=1)
+GDN_BLOCK = 64    # scan block of the tensor-core GDN kernel (tokens)
+SSD_BLOCK = 128   # scan block of the tensor-core SSD kernel (tokens)
+
+
+# ----------------------------------------------------------------------------- workload description
+
+def build_requests(name: str, rank: int = 0):
+    """List of requests: family, number of cached chunks K, context tokens, recompute tokens."""
+    if name == "cfg1":
+        return [dict(family="mamba2", K=8, total=8 * 1024, recompute=1024)]
+    if name == "cfg2":
+        return [dict(family="gdn", K=16, total=16 * 1024, recompute=int(0.2 * 16 * 1024))]
+    if name == "cfg3":
+        return [dict(family="gdn", K=32, total=32 * 1024, recompute=2048, shared_pool=True) for _ in range(8)]
+    if name == "cfg4":
+        return wl.ragged_mix(seed=4 + 1000 * rank)
+    raise ValueError(name)
+
+
+def gdn_scan_flops(tokens: int, s=GDN_SHAPE, C=GDN_BLOCK) -> float:
+    """Chunkwise GDN flops: per token and value head 2*(3 d_k d_v + 2 C d_v + 2 C d_k)
+    (K S, Q S, K^T U; the triangular solve applied to the right-hand side and P U; K K^T and Q K^T)."""
+    per = 2.0 * (3 * s["d_k"] * s["d_v"] + 2 * C * s["d_v"] + 2 * C * s["d_k"])
+    return per * s["H_v"] * tokens
+
+
+def ssd_scan_flops(tokens: int, s=SSD_SHAPE, Q=SSD_BLOCK) -> float:
+    """Chunkwise SSD flops: per token and head 2*(2 N P + Q P) plus C B^T once per group 2*Q*N."""
+    return (2.0 * (2 * s["N"] * s["P"] + Q * s["P"]) * s["H"] + 2.0 * Q * s["N"] * s["G"]) * tokens
+
+
+def gdn_scan_bytes(tokens: int, s=GDN_SHAPE) -> float:
+    return tokens * (2 * s["H_k"] * s["d_k"] * 2 + 2 * s["H_v"] * s["d_v"] * 2 + 2 * s["H_v"] * 4)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+class Family:
+    """Device-resident (and pinned-host) tensors of one recurrence family of the workload."""
+
+    def __init__(self, fam, reqs, seed, torch, b):
+        self.fam, self.reqs, self.torch, self.b = fam, reqs, torch, b
+        rng = np.random.default_rng(seed)
+        self.n_req = len(reqs)
+        shared = any(r.get("shared_pool") for r in reqs)
+        ks = [r["K"] for r in reqs]
+        self.cu_k = np.concatenate([[0], np.cumsum(ks)]).astype(np.int32)
+        if shared:
+            n_pool = ks[0]
+            self.ids = np.concatenate([wl.request_permutation(3, i, n_pool) for i in range(self.n_req)]).astype(np.int32)
+        else:
+            n_pool = int(self.cu_k[-1])
+            self.ids = np.arange(n_pool, dtype=np.int32)
+        lens = [r["recompute"] for r in reqs]
+        self.cu_seq = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        T = int(self.cu_seq[-1])
+        self.scan_tokens = T
+        self.context_tokens = int(sum(r["total"] for r in reqs))
+        bf = torch.bfloat16
+        h = {}
+        if fam == "gdn":
+            s = GDN_SHAPE
+            h["states"] = torch.from_numpy(wl.synthetic_states(rng, n_pool, s["H_v"], s["d_k"], s["d_v"]))
+            h["trans"] = torch.from_numpy(wl.cheap_gdn_transitions(rng, n_pool, s["H_v"], s["d_k"]))
+            tok = wl.gdn_tokens(rng, T, s["H_k"], s["H_v"], s["d_k"], s["d_v"], io="bf16")
+            for n in ("q", "k", "v"):
+                h[n] = torch.from_numpy(tok[n]).to(bf)
+            h["g"], h["beta"] = torch.from_numpy(tok["g"]), torch.from_numpy(tok["beta"])
+            self.family_code = b.LKV_FAMILY_GDN
+            self.state_shape = (s["H_v"], s["d_k"], s["d_v"])
+            self.out_shape = (T, s["H_v"], s["d_v"])
+        else:
+            s = SSD_SHAPE
+            h["states"] = torch.from_numpy(wl.synthetic_states(rng, n_pool, s["H"], s["N"], s["P"]))
+            h["trans"] = torch.from_numpy(wl.synthetic_logdecay(rng, n_pool, s["H"]))
+            h["A"] = torch.from_numpy(wl.ssd_A(rng, s["H"]))
+            tok = wl.ssd_tokens(rng, T, s["H"], s["P"], s["N"], s["G"], io="bf16")
+            for n in ("x", "B", "C"):
+                h[n] = torch.from_numpy(tok[n]).to(bf)
+            h["dt"] = torch.from_numpy(tok["dt"])
+            self.family_code = b.LKV_FAMILY_MAMBA2
+            self.state_shape = (s["H"], s["N"], s["P"])
+            self.out_shape = (T, s["H"], s["P"])
+        self.host = {n: t.contiguous().pin_memory() for n, t in h.items()}
+        self.dev = {n: t.cuda(non_blocking=True) for n, t in self.host.items()}
+        self.S0_last = torch.empty((self.n_req,) + self.state_shape, dtype=torch.float32, device="cuda")
+        self.S0 = torch.empty_like(self.S0_last)
+        self.S_T = torch.empty_like(self.S0_last)
+        self.out = torch.empty(self.out_shape, dtype=bf, device="cuda")
+        self.host_out = torch.empty(self.out_shape, dtype=bf).pin_memory()
+        self.host_S_T = torch.empty(self.S_T.shape, dtype=torch.float32).pin_memory()
+        self.ws_init = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+        self.ws_scan = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
+        self.d2h_bytes = self.host_out.numel() * 2 + self.host_S_T.numel() * 4
+        self.pool_bytes_unique = h["states"].numel() * 4 + h["trans"].numel() * 4
+        self.launches = 3
+
+    def upload(self):
+        for n, t in self.host.items():
+            self.dev[n].copy_(t, non_blocking=True)
+
+    def download(self):
+        self.host_out.copy_(self.out, non_blocking=True)
+        self.host_S_T.copy_(self.S_T, non_blocking=True)
+
+    def init_last(self):
+        b, d = self.b, self.dev
+        b.lkv_init_state_batched(d["states"], None, self.ids, self.cu_k, self.n_req, b.LKV_INIT_LAST, None,
+                                 self.S0_last, family=self.family_code, workspace_t=self.ws_init)
+
+    def init_exact(self):
+        b, d = self.b, self.dev
+        b.lkv_init_state_batched(d["states"], d["trans"], self.ids, self.cu_k, self.n_req, b.LKV_INIT_EXACT, None,
+                                 self.S0, family=self.family_code, workspace_t=self.ws_init)
+
+    def scan(self):
+        b, d = self.b, self.dev
+        if self.fam == "gdn":
+            b.lkv_gdn_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], self.S0, self.out, self.S_T,
+                          cu_seqlens=self.cu_seq, workspace_t=self.ws_scan)
+        else:
+            b.lkv_ssd_fwd(d["x"], d["dt"], d["A"], d["B"], d["C"], self.S0, self.out, self.S_T,
+                          cu_seqlens=self.cu_seq, workspace_t=self.ws_scan)
+
+    def step(self):
+        self.init_last()
+        self.init_exact()
+        self.scan()
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def cpu_baseline_sample(seconds_hint: float = 15.0):
+    """The oracle as it stands, timed on this machine's cores on a bounded sample of the workload:
+    exact composition of one GDN request (K = 16) plus a 12288-token GDN scan, all 32 value heads,
+    and the same for one Mamba-2 request (K = 16, 12288 tokens, 80 heads)."""
+    import oracle
+    rng = np.random.default_rng(99)
+    s, m = GDN_SHAPE, SSD_SHAPE
+    T, K = 12288, 16
+    tok = wl.gdn_tokens(rng, T, s["H_k"], s["H_v"], s["d_k"], s["d_v"])
+    states = wl.synthetic_states(rng, K, s["H_v"], s["d_k"], s["d_v"])
+    trans = wl.cheap_gdn_transitions(rng, K, s["H_v"], s["d_k"])
+    mt = wl.ssd_tokens(rng, T, m["H"], m["P"], m["N"], m["G"])
+    A = wl.ssd_A(rng, m["H"])
+    mstates = wl.synthetic_states(rng, K, m["H"], m["N"], m["P"])
+    lam = wl.synthetic_logdecay(rng, K, m["H"])
+    oracle.num_threads()
+    t0 = time.perf_counter()
+    S0 = oracle.init_exact_gdn(states, trans)
+    oracle.gdn_seq(tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], S0)
+    M0 = oracle.init_exact_mamba(mstates, lam)
+    oracle.ssd_seq(mt["x"], mt["dt"], A, mt["B"], mt["C"], M0)
+    dt = time.perf_counter() - t0
+    # context covered by the sample at the workload's recompute ratio (0.2): each request's
+    # T recomputed tokens stand for T / 0.2 context tokens
+    context = 2 * T / 0.2
+    return dict(value=context / dt, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
+                sample=f"1 GDN + 1 Mamba-2 request, K={K} exact composition + {T}-token scan each "
+                       f"(= {int(context)} context tokens at r=0.2), {dt:.2f} s"), dt
+
+
+def run_reference(args):
+    """--impl reference: the fp64 oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        cpu_baseline_sample()
+    times, base = [], None
+    for _ in range(args.steps):
+        base, dt = cpu_baseline_sample()
+        times.append(dt)
+    context = 2 * 12288 / 0.2
+    t = sum(times) / len(times)
+    value = context / t
+    base["value"] = value
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * t, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", config={"workload": args.workload, "sample": base["sample"]},
+                cpu_baseline=base, e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_11231_b200 import binding as b
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    b.load()
+
+    reqs = build_requests(args.workload, rank)
+    fams = []
+    for fam in ("mamba2", "gdn"):
+        sub = [r for r in reqs if r["family"] == fam]
+        if sub:
+            fams.append(Family(fam, sub, seed=100 + rank * 10 + len(fams), torch=torch, b=b))
+    torch.cuda.synchronize()
+    context_tokens = sum(f.context_tokens for f in fams)
+    scan_tokens = sum(f.scan_tokens for f in fams)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def timed(fn, steps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for _ in range(steps):
+            fn()
+        ev1.record()
+        barrier()
+        return max_over_ranks(ev0.elapsed_time(ev1) / steps)  # ms per step
+
+    def step():
+        for f in fams:
+            f.step()
+
+    def step_e2e():
+        for f in fams:
+            f.upload()
+            f.step()
+            f.download()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed(step, args.steps)
+    # per-kernel device times over the same K steps (each kernel timed alone, inputs far larger than L2)
+    parts = {}
+    for f in fams:
+        for name, fn in (("init_last", f.init_last), ("init_exact", f.init_exact), ("scan", f.scan)):
+            parts[f"{f.fam}.{name}"] = timed(fn, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    e2e_steps = max(1, min(args.steps, 3))
+    step_e2e()
+    ms_e2e = timed(step_e2e, e2e_steps)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = {}
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            peaks = json.load(fh)
+        peak_src = "measured"
+    except OSError:
+        peaks = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+        peak_src = "fallback"
+
+    # dominant kernel: the scan of the family with the larger share of the step
+    dom = max(parts, key=parts.get)
+    fam_name, kern = dom.split(".")
+    f = next(x for x in fams if x.fam == fam_name)
+    if kern == "scan":
+        flops = gdn_scan_flops(f.scan_tokens) if fam_name == "gdn" else ssd_scan_flops(f.scan_tokens)
+        achieved = flops / (parts[dom] * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"] if parts[dom] > 50.0 else peaks["bf16_tflops"]
+        roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                    kernel=dom, peak_source=peak_src)
+    else:
+        nbytes = f.pool_bytes_unique + f.S0.numel() * 4
+        achieved = nbytes / (parts[dom] * 1e-3) / 1e9
+        roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], traffic=None, kernel=dom, peak_source=peak_src)
+
+    detail = {}
+    for f in fams:
+        t_scan = parts[f"{f.fam}.scan"] * 1e-3
+        flops = gdn_scan_flops(f.scan_tokens) if f.fam == "gdn" else ssd_scan_flops(f.scan_tokens)
+        comp_bytes = f.pool_bytes_unique + f.S0.numel() * 4
+        detail[f.fam] = dict(
+            requests=f.n_req, context_tokens=f.context_tokens, scan_tokens=f.scan_tokens,
+            init_last_us=1e3 * parts[f"{f.fam}.init_last"], init_exact_us=1e3 * parts[f"{f.fam}.init_exact"],
+            scan_us=1e3 * parts[f"{f.fam}.scan"], scan_tokens_per_s=f.scan_tokens / t_scan,
+            scan_tflops=flops / t_scan / 1e12,
+            compose_gbs_unique=comp_bytes / (parts[f"{f.fam}.init_exact"] * 1e-3) / 1e9,
+            compose_frac_of_hbm=comp_bytes / (parts[f"{f.fam}.init_exact"] * 1e-3) / 1e9 / peaks["hbm_gbs"])
+
+    base, _ = cpu_baseline_sample() if world == 1 else (None, None)
+    line = dict(
+        metric=METRIC, value=world * context_tokens / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
+        warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16", data="synthetic",
+        config=dict(workload=args.workload, requests=len(reqs), context_tokens=context_tokens,
+                    scan_tokens=scan_tokens, l2="inputs larger than L2 (no flush needed)" if
+                    sum(f.h2d_bytes for f in fams) > 512e6 else "inputs smaller than L2: warm-cache numbers",
+                    sharding="requests across ranks, no collective"),
+        e2e=dict(value=world * context_tokens / (ms_e2e * 1e-3), unit=UNIT,
+                 h2d_bytes_per_step=sum(f.h2d_bytes for f in fams), d2h_bytes_per_step=sum(f.d2h_bytes for f in fams),
+                 ms_per_step=ms_e2e, steps=e2e_steps),
+        gpu_launches=sum(f.launches for f in fams) * args.steps,
+        scan_tokens_per_s=world * scan_tokens / (ms * 1e-3),
+        roofline=roof, kernels=detail, clocks=clocks)
+    if base is not None:
+        line["cpu_baseline"] = base
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
