@@ -334,3 +334,24 @@ def test_config0_whole_path():
         o, ST = _run_gdn(suffix, S0_ex[None], "f32")
         n_pre = cfg["K"] * cfg["chunk_len"]
         assert maxrel(o, o_all[n_pre:]) <= TOL_F32 and maxrel(ST[0], ST_all) <= TOL_F32
+
+
+def test_batched_init_with_index_list_in_workspace():
+    """More chunk ids than fit in the kernel parameters: the list travels through the workspace."""
+    rng = np.random.default_rng(21)
+    n, H, N, P = 24, 2, 16, 32
+    pool = wl.synthetic_states(rng, n, H, N, P)
+    lam = wl.synthetic_logdecay(rng, n, H, lo=-0.5)
+    n_req, K = 160, 30
+    ids = rng.integers(0, n, size=n_req * K).astype(np.int32)
+    cu = (np.arange(n_req + 1) * K).astype(np.int32)
+    assert ids.size + 2 * n_req + 1 > 4000
+    got = host(b.lkv_init_state_batched(dev(pool), dev(lam), ids, cu, n_req, b.LKV_INIT_EXACT, None,
+                                        family=b.LKV_FAMILY_MAMBA2))
+    for r in (0, 1, 77, n_req - 1):
+        assert maxrel(got[r], oracle.init_exact_mamba(pool, lam, ids[cu[r]:cu[r + 1]])) <= 1e-5
+    sel = rng.integers(0, K, size=n_req).astype(np.int32)
+    got = host(b.lkv_init_state_batched(dev(pool), None, ids, cu, n_req, b.LKV_INIT_INDEX, sel,
+                                        family=b.LKV_FAMILY_MAMBA2))
+    for r in (0, 5, n_req - 1):
+        assert got[r].tobytes() == pool[ids[cu[r] + sel[r]]].tobytes()
