@@ -199,6 +199,42 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
                            const lkv_init_desc *d, void *stream);
 
 /*
+ * lkv_init_state_batched without any caller-provided scratch.  (The paper has no
+ * counterpart: this entry point exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where device memory cannot be allocated or handed
+ * over -- a serving engine that has already given its whole memory budget to its own
+ * pool and forbids cudaMalloc on the request path, a plugin called from inside
+ * someone else's allocator-owned stream callback, a process that must not touch the
+ * allocator while another component is capturing work.  Such a caller still owns the
+ * inputs and the output, but has nowhere to get a workspace from.
+ *
+ * What differs from lkv_init_state_batched: d->workspace and d->workspace_bytes are
+ * ignored.  The scratch the batched kernels use (status word + the request/chunk index
+ * list) lives in a fixed array inside the library image, LKV_STATIC_SCRATCH_BYTES
+ * bytes of device memory on every GPU that loads the library, held until the process
+ * exits.  The call allocates nothing and frees nothing, directly or through a library.
+ *
+ * Limits and rules:
+ *   - 2 * n_req + 1 + (number of chunk ids) must not exceed LKV_STATIC_MAX_INDEX;
+ *     a larger request returns LKV_ERR_WORKSPACE and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array; it keeps whatever the previous
+ *     call left in it, and every call rewrites the parts it reads before its kernel
+ *     runs.  Two calls that can overlap on the GPU (different streams, no ordering
+ *     between them) race on it: order them, or use lkv_init_state_batched with
+ *     separate workspaces.
+ *   - Everything else (arguments, modes, errors, results) is as for
+ *     lkv_init_state_batched; results are identical bit for bit.
+ */
+#define LKV_STATIC_MAX_INDEX 16384
+#define LKV_STATIC_SCRATCH_BYTES (256 + 4 * LKV_STATIC_MAX_INDEX)
+int lkv_init_state_batched_static(const void *states, const void *transitions, const int32_t *chunk_ids,
+                                  const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index,
+                                  void *S0, const lkv_init_desc *d, void *stream);
+
+/*
  * Gated DeltaNet scan from an initial state (Eq. 1 with Eq. 3; Algorithm 1, line 3).
  * For each sequence and value head, in token order:
  *     S_t = exp(g_t) (I - beta_t k_t k_t^T) S_{t-1} + beta_t k_t v_t^T

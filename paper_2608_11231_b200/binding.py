@@ -27,7 +27,7 @@ LKV_INIT_LAST, LKV_INIT_INDEX, LKV_INIT_EXACT = 0, 1, 2
 LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
 LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
-EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_gdn_fwd", "lkv_ssd_fwd",
+EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
            "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
 
 
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
         vp, ci = ctypes.c_void_p, ctypes.c_int
         lib.lkv_init_state.argtypes = [vp, vp, ci, ci, vp, ctypes.POINTER(lkv_init_desc), vp]
         lib.lkv_init_state_batched.argtypes = [vp, vp, vp, vp, ci, ci, vp, vp, ctypes.POINTER(lkv_init_desc), vp]
+        lib.lkv_init_state_batched_static.argtypes = lib.lkv_init_state_batched.argtypes
+        lib.lkv_init_state_batched_static.restype = ci
         lib.lkv_gdn_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), vp]
         lib.lkv_ssd_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_workspace_bytes.argtypes = [ci, vp, ci, ci]
@@ -188,6 +190,31 @@ def lkv_init_state_batched(states: torch.Tensor, transitions: Optional[torch.Ten
                                        _hp(sel), _ptr(S0), ctypes.byref(d), _stream(stream))
     if st != LKV_OK:
         raise LkvError(st, "lkv_init_state_batched")
+    return S0
+
+
+LKV_STATIC_MAX_INDEX = 16384
+
+
+def lkv_init_state_batched_static(states: torch.Tensor, transitions: Optional[torch.Tensor], chunk_ids, cu_k,
+                                  n_req: int, mode: int, sel_index=None, S0: Optional[torch.Tensor] = None, *,
+                                  family: int, compute: int = LKV_COMPUTE_AUTO, stream=None):
+    """lkv_init_state_batched for callers that cannot allocate: no workspace is passed or created.
+
+    The library keeps its scratch in a fixed array of its own (see the header for the size limit, the
+    first-call rule and why overlapping calls race).  Pass S0 to keep this wrapper allocation-free too;
+    if it is None the wrapper creates the output tensor, which a caller that cannot allocate would not do.
+    """
+    ids, cu, sel = _host_i32(chunk_ids), _host_i32(cu_k), _host_i32(sel_index)
+    n, H, d_k, d_v = states.shape
+    d = lkv_init_desc(family=family, H=H, d_k=d_k, d_v=d_v, n_chunks=n, state_dtype=_dtype_code(states),
+                      sel_index=0, compute=compute, chunk_ids=None, workspace=None, workspace_bytes=0)
+    if S0 is None:
+        S0 = torch.empty((n_req,) + tuple(states.shape[1:]), dtype=torch.float32, device=states.device)
+    st = load().lkv_init_state_batched_static(_ptr(states), _ptr(transitions), _hp(ids), _hp(cu), int(n_req),
+                                              int(mode), _hp(sel), _ptr(S0), ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_init_state_batched_static")
     return S0
 
 

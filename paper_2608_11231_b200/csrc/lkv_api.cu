@@ -294,3 +294,59 @@ const char *lkv_status_string(int status) {
 int lkv_version(void) { return LKV_VERSION; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Batched state initialisation for callers that cannot allocate device memory and therefore
+// have no workspace to pass (an engine whose allocator is closed on the request path, a
+// plugin running inside another component's memory budget).  The scratch is this fixed array,
+// part of the library image on every GPU that loads it.
+//
+// In host code the name `g_static_scratch` is only a handle for the runtime, NOT a device
+// address: the address a kernel may use has to be asked for with cudaGetSymbolAddress, once
+// per device and with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[LKV_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices];  // per device, filled on the first call there
+
+// Device address of the static scratch on the current device (nullptr on failure).
+void *static_scratch_for_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    void *p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);
+    }
+    return p;
+}
+}  // namespace
+
+extern "C" int lkv_init_state_batched_static(const void *states, const void *transitions, const int32_t *chunk_ids,
+                                             const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index,
+                                             void *S0, const lkv_init_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (n_req < 0) return LKV_ERR_DIM;
+    if (!cu_k) return LKV_ERR_NULL;
+    // size check first: beyond the fixed array there is nowhere to put the index list
+    const long long n_ints = 2LL * n_req + 1 + (cu_k[n_req] > 0 ? cu_k[n_req] : 0);
+    if (n_ints > LKV_STATIC_MAX_INDEX) return LKV_ERR_WORKSPACE;
+    void *scratch = static_scratch_for_current_device();
+    if (!scratch) return LKV_ERR_CUDA;
+    // the array keeps the previous call's contents: the status word must start at zero
+    if (cudaMemsetAsync(scratch, 0, kWsHeaderBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    lkv_init_desc local = *d;
+    local.workspace = scratch;
+    local.workspace_bytes = LKV_STATIC_SCRATCH_BYTES;
+    return init_impl(states, transitions, chunk_ids, cu_k, n_req, mode, sel_index, S0, &local, stream);
+}
