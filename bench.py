@@ -290,15 +290,52 @@ def run_ours(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
 
-    def timed(fn, steps):
+    total_input_bytes = sum(f.h2d_bytes for f in fams)
+    cold_by_size = total_input_bytes > 4 * 126e6        # inputs far larger than the 126 MB L2
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+
+    def flush_l2():
+        flush_buf.zero_()
+
+    def graph_of(fn):
+        """Capture fn (launches only, no allocation) into a CUDA graph so that host overhead of the
+        Python binding does not enter device timings of microsecond-scale kernels."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g
+
+    def timed_back_to_back(replay, steps):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         ev0.record()
         for _ in range(steps):
-            fn()
+            replay()
         ev1.record()
         barrier()
         return max_over_ranks(ev0.elapsed_time(ev1) / steps)  # ms per step
+
+    def timed_flushed(replay, steps, reduce="mean"):
+        """Each iteration timed alone, L2 flushed (untimed) before it."""
+        ts = []
+        barrier()
+        for _ in range(steps):
+            flush_l2()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            replay()
+            ev1.record()
+            ev1.synchronize()
+            ts.append(ev0.elapsed_time(ev1))
+        barrier()
+        t = statistics.median(ts) if reduce == "median" else sum(ts) / len(ts)
+        return max_over_ranks(t)
 
     def step():
         for f in fams:
@@ -312,19 +349,26 @@ def run_ours(args):
 
     for _ in range(max(args.warmup, 3)):
         step()
+    g_step = graph_of(step)
+    for _ in range(max(args.warmup, 3)):
+        g_step.replay()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(step, args.steps)
-    # per-kernel device times over the same K steps (each kernel timed alone, inputs far larger than L2)
+    if cold_by_size:
+        ms = timed_back_to_back(g_step.replay, args.steps)
+    else:
+        ms = timed_flushed(g_step.replay, args.steps)
+    # per-kernel device times: each kernel alone in its own graph, L2 flushed before every launch, median
     parts = {}
     for f in fams:
         for name, fn in (("init_last", f.init_last), ("init_exact", f.init_exact), ("scan", f.scan)):
-            parts[f"{f.fam}.{name}"] = timed(fn, args.steps)
+            g = graph_of(fn)
+            parts[f"{f.fam}.{name}"] = timed_flushed(g.replay, max(args.steps, 5), reduce="median")
     clocks = sampler.stop() if rank == 0 else None
     e2e_steps = max(1, min(args.steps, 3))
     step_e2e()
-    ms_e2e = timed(step_e2e, e2e_steps)
+    ms_e2e = timed_back_to_back(step_e2e, e2e_steps)
 
     if rank != 0:
         if world > 1:
@@ -375,8 +419,8 @@ def run_ours(args):
         warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="bf16", data="synthetic",
         config=dict(workload=args.workload, requests=len(reqs), context_tokens=context_tokens,
-                    scan_tokens=scan_tokens, l2="inputs larger than L2 (no flush needed)" if
-                    sum(f.h2d_bytes for f in fams) > 512e6 else "inputs smaller than L2: warm-cache numbers",
+                    scan_tokens=scan_tokens, l2="inputs far larger than L2, steps timed back to back" if cold_by_size else
+                    "L2 flushed (512 MiB write, untimed) before every timed step", timing="CUDA-graph replay, CUDA events",
                     sharding="requests across ranks, no collective"),
         e2e=dict(value=world * context_tokens / (ms_e2e * 1e-3), unit=UNIT,
                  h2d_bytes_per_step=sum(f.h2d_bytes for f in fams), d2h_bytes_per_step=sum(f.d2h_bytes for f in fams),

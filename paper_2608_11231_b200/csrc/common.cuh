@@ -48,7 +48,7 @@ struct InitArgs {
     const void *states;        // pool
     const float *transitions;  // pool (log-decay or dense)
     float *S0;                 // [n_req, H, d_k, d_v]
-    int32_t n_req, H, d_k, d_v;
+    int32_t n_req, H, d_k, d_v, n_chunks;
     int32_t off_sel;           // offset of sel[n_req] in idx, or -1 (= last block)
     int32_t off_ids;           // offset of ids[total_K] in idx; cu_k[n_req + 1] sits at 0
     int32_t *status;           // device status word

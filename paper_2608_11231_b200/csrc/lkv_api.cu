@@ -89,6 +89,7 @@ int init_impl(const void *states, const void *transitions, const int32_t *chunk_
     a.H = d->H;
     a.d_k = d->d_k;
     a.d_v = d->d_v;
+    a.n_chunks = d->n_chunks;
     a.status = static_cast<int32_t *>(d->workspace);
     std::vector<int32_t> ints;
     ints.reserve(n_ints);

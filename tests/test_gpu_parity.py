@@ -355,3 +355,24 @@ def test_batched_init_with_index_list_in_workspace():
                                         family=b.LKV_FAMILY_MAMBA2))
     for r in (0, 5, n_req - 1):
         assert got[r].tobytes() == pool[ids[cu[r] + sel[r]]].tobytes()
+
+
+def test_gdn_exact_tensor_many_heads_ragged():
+    """Enough (request, head) pairs that the tensor-core kernel takes its wide column blocks; ragged K
+    including the K = 1 identity and the empty request; the device status word must stay clean."""
+    rng = np.random.default_rng(44)
+    n, H, dk, dv = 10, 8, 128, 128
+    pool = wl.synthetic_states(rng, n, H, dk, dv)
+    trans = wl.synthetic_gdn_transitions(rng, n, H, dk)
+    ks = [4, 1, 0, 9, 2, 3, 7, 5]
+    cu = np.concatenate([[0], np.cumsum(ks)]).astype(np.int32)
+    ids = np.concatenate([rng.integers(0, n, size=k) for k in ks]).astype(np.int32)
+    ws = _torch().zeros(4096, dtype=_torch().uint8, device="cuda")
+    got = host(b.lkv_init_state_batched(dev(pool), dev(trans), ids, cu, len(ks), b.LKV_INIT_EXACT, None,
+                                        family=b.LKV_FAMILY_GDN, compute=b.LKV_COMPUTE_TENSOR, workspace_t=ws))
+    assert b.lkv_device_status(ws) == b.LKV_OK
+    for r, k in enumerate(ks):
+        ref = oracle.init_exact_gdn(pool, trans, ids[cu[r]:cu[r + 1]])
+        assert maxrel(got[r], ref) <= 2e-3, (r, k, maxrel(got[r], ref))
+    assert got[1].tobytes() == pool[ids[cu[1]]].tobytes()
+    assert not got[2].any()
