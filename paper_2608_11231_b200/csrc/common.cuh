@@ -63,7 +63,7 @@ struct GdnArgs {
     const float *g, *beta, *S0;
     void *o;
     float *S_T;
-    int32_t n_seq, H_k, H_v, d_k, d_v;
+    int32_t n_seq, T_total, H_k, H_v, d_k, d_v;
     float scale;
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
@@ -74,7 +74,7 @@ struct SsdArgs {
     const float *dt, *A, *S0;
     void *y;
     float *S_T;
-    int32_t n_seq, H, P, N, G;
+    int32_t n_seq, T_total, H, P, N, G;
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
 };

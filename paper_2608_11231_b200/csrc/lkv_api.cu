@@ -188,7 +188,7 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
 
     GdnArgs a;
     a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = S_T;
-    a.n_seq = d->n_seq; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
+    a.n_seq = d->n_seq; a.T_total = d->T_total; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
     a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
@@ -231,7 +231,7 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
 
     SsdArgs a;
     a.x = x; a.dt = dt; a.A = A; a.B = B; a.C = C; a.S0 = S0; a.y = y; a.S_T = S_T;
-    a.n_seq = d->n_seq; a.H = d->H; a.P = d->P; a.N = d->N; a.G = d->G;
+    a.n_seq = d->n_seq; a.T_total = d->T_total; a.H = d->H; a.P = d->P; a.N = d->N; a.G = d->G;
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
     const bool tensor_fits = ssd_scan_tensor_supported(a, io_bf16);

@@ -1,6 +1,386 @@
-// SSD scan on tensor cores (placeholder until the tcgen05 kernel lands).
+// Chunkwise Mamba-2 (SSD) scan on the 5th-generation tensor cores (Eq. 1 with Eq. 2), for
+// headdim P = 64, d_state N = 128 and bf16 x/B/C/y.  One CTA owns one (sequence, head) and walks
+// the sequence in blocks of 128 tokens with the N x P state carried on chip (fp32 in tensor memory,
+// a bf16 copy in shared memory as an MMA operand).  With l the running sum of dt * A_h inside the
+// block and S the incoming state, per block:
+//   (a) G      = C B^T                                   [128 x 128], K = N                 tcgen05
+//       G'_ti  = G_ti e^{l_t - l_i} dt_i  (i <= t), 0 otherwise -> bf16 operand             epilogue warps
+//   (b) Yintra = G' X                                    [128 x 64],  K = 128 tokens         tcgen05
+//   (c) Yinter = C S                                     [128 x 64],  K = N                  tcgen05
+//       y_t    = Yintra_t + e^{l_t} Yinter_t                                                 epilogue warps
+//   (d) S     <- e^{l_Q} S + B^T X~,  X~_i = e^{l_Q - l_i} dt_i x_i   [128 x 64], K = tokens   tcgen05
+//       (the state is pre-scaled in tensor memory, (d) accumulates onto it)                  state warps
+// Only (c) depends on the previous block, so the tensor pipe and the SIMT warps overlap freely;
+// the block-to-block chain is (d) -> state copy -> (c).  A padded token has dt = 0.
+// Warps 0-7 epilogue (thread = token row, warpgroup = column half), 8-11 state and per-block
+// scalars, 12 TMA, 13 MMA issue.  All waits on mbarriers are bounded.
 #include "common.cuh"
+#include "tc_common.cuh"
+
 namespace lkv {
-bool ssd_scan_tensor_supported(const SsdArgs &, bool) { return false; }
-cudaError_t launch_ssd_scan_tensor(const SsdArgs &, cudaStream_t) { return cudaErrorNotSupported; }
+
+namespace {
+
+using namespace tc;
+
+constexpr int kP = 64;     // headdim
+constexpr int kN = 128;    // d_state
+constexpr int kQ = 128;    // tokens per block
+constexpr int kThreads = 448;
+
+// shared-memory map (bytes, after 1024-byte alignment); every tile row is 128 bytes, 128-byte swizzle
+constexpr int kXTile = kQ * 128;            // X [128 tokens x 64 p]
+constexpr int kBTile = 2 * kQ * 128;        // B [B_kb0 | B_kb1], each [128 tokens x 64 n]
+constexpr int kCTile = 2 * kQ * 128;        // C likewise; reused for G' once (a) and (c) are done
+constexpr int kStageBytes = kXTile + kBTile + kCTile;   // 80 KB
+constexpr int kOffX2 = 2 * kStageBytes;     // X~ [128 tokens x 64 p]
+constexpr int kOffHb = kOffX2 + kXTile;     // bf16 state [128 n x 64 p]
+constexpr int kOffSc = kOffHb + kN * 128;   // per-block scalars, double-buffered
+constexpr int kScFloats = 4 * kQ;           // l, e^{l}, s = e^{l_Q - l} dt, dt
+constexpr int kSmemBytes = kOffSc + 2 * kScFloats * 4 + 1024;
+
+// tensor-memory map (columns)
+constexpr uint32_t kTmG = 0;        // 128
+constexpr uint32_t kTmYa = 128;     // Yintra, 2 x 64
+constexpr uint32_t kTmYe = 256;     // Yinter, 2 x 64
+constexpr uint32_t kTmH = 384;      // 64
+constexpr uint32_t kTmemCols = 512;
+
+struct Bars {
+    uint64_t full[2], tiles_free[2];
+    uint64_t ac_done, y_done, h_done;                  // tcgen05.commit targets
+    uint64_t mg_ready, yo_done[2];                     // 256 epilogue threads
+    uint64_t sc_ready[2], x2_ready, hb_ready;          // 128 state threads
+};
+
+__device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred P1;\n\telect.sync _|P1, %1;\n\tselp.u32 %0, 1, 0, P1;\n\t}" : "=r"(e) : "r"(0xffffffffu));
+    return e;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant__ CUtensorMap mapX,
+                       const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    __shared__ Bars bars;
+    __shared__ uint32_t tmem_base;
+    __shared__ int dead;
+    __shared__ float scan_carry[4];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.x, seq = blockIdx.y;
+    const int grp = h / (a.H / a.G);
+    const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
+    const int nblk = (t_end - t_begin + kQ - 1) / kQ;
+    const size_t sbase = (static_cast<size_t>(seq) * a.H + h) * kN * kP;
+
+    if (nblk == 0) {  // empty sequence: hand the state through untouched
+        if (a.S_T && a.S_T != a.S0)
+            for (int e = tid; e < kN * kP; e += kThreads) a.S_T[sbase + e] = a.S0 ? a.S0[sbase + e] : 0.f;
+        return;
+    }
+    if (tid == 0) {
+        dead = 0;
+        uint64_t *b1 = &bars.full[0];
+        for (int i = 0; i < 7; ++i) mbar_init(b1 + i, 1);
+        uint64_t *b256 = &bars.mg_ready;
+        for (int i = 0; i < 3; ++i) mbar_init(b256 + i, 256);
+        uint64_t *b128 = &bars.sc_ready[0];
+        for (int i = 0; i < 4; ++i) mbar_init(b128 + i, 128);
+        mbar_fence_init();
+    }
+    if (warp == 13) tmem_alloc(&tmem_base, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tm = tmem_base;
+    float *scal = reinterpret_cast<float *>(sm + kOffSc);
+
+    if (warp == 12) {
+        // ======================================================= TMA producer
+        if (lane == 0) {
+            tma_prefetch_desc(&mapX);
+            tma_prefetch_desc(&mapB);
+            tma_prefetch_desc(&mapC);
+            for (int b = 0; b < nblk; ++b) {
+                const int st = b & 1;
+                if (b >= 2) mbar_wait(&bars.tiles_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                unsigned char *base = sm + st * kStageBytes;
+                const int row = t_begin + b * kQ;
+                mbar_expect_tx(&bars.full[st], kStageBytes);
+                tma_load_2d(base, &mapX, h * kP, row, &bars.full[st]);
+                for (int kb = 0; kb < 2; ++kb) {
+                    tma_load_2d(base + kXTile + kb * kQ * 128, &mapB, grp * kN + kb * 64, row, &bars.full[st]);
+                    tma_load_2d(base + kXTile + kBTile + kb * kQ * 128, &mapC, grp * kN + kb * 64, row, &bars.full[st]);
+                }
+            }
+        }
+    } else if (warp == 13) {
+        // ======================================================= MMA issuer (one elected thread)
+        if (elect_one()) {
+            constexpr uint32_t idA = umma_idesc(kFmtBF16, false, false, 128, 128);   // (a): C, B both K-major
+            constexpr uint32_t idC = umma_idesc(kFmtBF16, false, true, 128, 64);     // (c), (b): B operand MN-major
+            constexpr uint32_t idD = umma_idesc(kFmtBF16, true, true, 128, 64);      // (d): both MN-major
+            const uint64_t dHb = umma_desc(smem_u32(sm + kOffHb), 0, 1024);
+            const uint64_t dX2 = umma_desc(smem_u32(sm + kOffX2), 0, 1024);
+            for (int b = 0; b < nblk; ++b) {
+                const uint32_t par = b & 1;
+                const uint32_t sbase_u = smem_u32(sm + (b & 1) * kStageBytes);
+                const uint64_t dX = umma_desc(sbase_u, 0, 1024);
+                const uint64_t dBk = umma_desc(sbase_u + kXTile, 0, 1024);                 // B tile, K-major view
+                const uint64_t dBm = umma_desc(sbase_u + kXTile, kQ * 128, 1024);          // B tile, MN-major view (n blocks 16 KB apart)
+                const uint64_t dCk = umma_desc(sbase_u + kXTile + kBTile, 0, 1024);        // C tile, later G'
+                mbar_wait(&bars.full[b & 1], (b >> 1) & 1, &dead, a.status);
+                mbar_wait(&bars.hb_ready, par, &dead, a.status);
+                if (b >= 2) mbar_wait(&bars.yo_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+                tc_fence_after_sync();
+                // (c) Yinter = C S : A = C (K = n), B = bf16 state read MN-major (rows = n)
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tm + kTmYe + 64 * par, dCk + (((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4), dHb + ((k * 16 * 128) >> 4), idC, k > 0);
+                // (a) G = C B^T
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint64_t off = ((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4;
+                    umma_bf16(tm + kTmG, dCk + off, dBk + off, idA, k > 0);
+                }
+                umma_commit(&bars.ac_done);
+                // (d) S += B^T X~ : A = B tile read MN-major (rows = tokens), B = X~ read MN-major
+                mbar_wait(&bars.x2_ready, par, &dead, a.status);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tm + kTmH, dBm + ((k * 16 * 128) >> 4), dX2 + ((k * 16 * 128) >> 4), idD, true);
+                umma_commit(&bars.h_done);
+                // (b) Yintra = G' X : A = G' (in the C buffer, K = tokens), B = X read MN-major
+                mbar_wait(&bars.mg_ready, par, &dead, a.status);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tm + kTmYa + 64 * par, dCk + (((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4), dX + ((k * 16 * 128) >> 4), idC, k > 0);
+                umma_commit(&bars.y_done);
+                umma_commit(&bars.tiles_free[b & 1]);
+            }
+        }
+    } else if (warp >= 8) {
+        // ======================================================= state warpgroup: thread = token (scalars, X~) / state row n
+        const int x = tid - 256;   // 0..127
+        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const float Ah = a.A[h];
+        auto prepare_scalars = [&](int b) {
+            float *dst = scal + (b & 1) * kScFloats;
+            const int t = t_begin + b * kQ + x;
+            const float dtv = (t < t_end) ? a.dt[static_cast<size_t>(t) * a.H + h] : 0.f;
+            float run = dtv * Ah;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float up = __shfl_up_sync(0xffffffffu, run, o);
+                if (lane >= o) run += up;
+            }
+            if (lane == 31) scan_carry[warp & 3] = run;
+            named_bar_sync(1, 128);
+            for (int w = 0; w < (warp & 3); ++w) run += scan_carry[w];
+            dst[x] = run;
+            dst[kQ + x] = __expf(run);
+            named_bar_sync(1, 128);
+            dst[2 * kQ + x] = __expf(dst[kQ - 1] - run) * dtv;
+            dst[3 * kQ + x] = dtv;
+            named_bar_sync(1, 128);
+            mbar_arrive(&bars.sc_ready[b & 1]);
+        };
+        prepare_scalars(0);
+        // initial state: fp32 into tensor memory pre-scaled by e^{l_Q} of block 0, bf16 copy unscaled
+        {
+            const float gq = scal[kQ + kQ - 1];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint32_t rr[32], sc[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float v = a.S0 ? a.S0[sbase + static_cast<size_t>(x) * kP + 32 * q + c] : 0.f;
+                    rr[c] = __float_as_uint(v);
+                    sc[c] = __float_as_uint(v * gq);
+                }
+                tmem_st32(lane_base + kTmH + 32 * q, sc);
+#pragma unroll
+                for (int c8 = 0; c8 < 4; ++c8) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) w[e] = pack_bf16(__uint_as_float(rr[8 * c8 + 2 * e]), __uint_as_float(rr[8 * c8 + 2 * e + 1]));
+                    *reinterpret_cast<uint4 *>(sm + kOffHb + sw128_offset(x, 4 * q + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            tmem_st_wait();
+            fence_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars.hb_ready);
+        }
+        for (int b = 0; b < nblk; ++b) {
+            const float *sc = scal + (b & 1) * kScFloats;
+            // X~ row of token x: s_x * X[x][:]
+            mbar_wait(&bars.full[b & 1], (b >> 1) & 1, &dead, a.status);
+            {
+                const unsigned char *xt = sm + (b & 1) * kStageBytes;
+                const float s = sc[2 * kQ + x];
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    const uint32_t off = sw128_offset(x, c8);
+                    const uint4 v = *reinterpret_cast<const uint4 *>(xt + off);
+                    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        w[e] = pack_bf16(__uint_as_float(in[e] << 16) * s, __uint_as_float(in[e] & 0xFFFF0000u) * s);
+                    *reinterpret_cast<uint4 *>(sm + kOffX2 + off) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            fence_async_smem();
+            mbar_arrive(&bars.x2_ready);
+            if (b + 1 < nblk) {
+                // the scalar buffer of block b+1 is the one block b-1 used: its outputs must be written
+                if (b >= 1) mbar_wait(&bars.yo_done[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
+                prepare_scalars(b + 1);
+            }
+            // state after (d): copy for the next block's (c), pre-scale for its (d); or S_T at the end
+            mbar_wait(&bars.h_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            const bool last = b + 1 == nblk;
+            const float gq = last ? 1.f : scal[((b + 1) & 1) * kScFloats + kQ + kQ - 1];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                uint32_t rr[32];
+                tmem_ld32(lane_base + kTmH + 32 * q, rr);
+                tmem_ld_wait();
+                if (last) {
+                    if (a.S_T) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            *reinterpret_cast<float4 *>(a.S_T + sbase + static_cast<size_t>(x) * kP + 32 * q + c) =
+                                make_float4(__uint_as_float(rr[c]), __uint_as_float(rr[c + 1]), __uint_as_float(rr[c + 2]), __uint_as_float(rr[c + 3]));
+                    }
+                } else {
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) w[e] = pack_bf16(__uint_as_float(rr[8 * c8 + 2 * e]), __uint_as_float(rr[8 * c8 + 2 * e + 1]));
+                        *reinterpret_cast<uint4 *>(sm + kOffHb + sw128_offset(x, 4 * q + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) rr[c] = __float_as_uint(__uint_as_float(rr[c]) * gq);
+                    tmem_st32(lane_base + kTmH + 32 * q, rr);
+                }
+            }
+            if (!last) {
+                tmem_st_wait();
+                fence_async_smem();
+                tc_fence_before_sync();
+                mbar_arrive(&bars.hb_ready);
+            }
+        }
+    } else {
+        // ======================================================= epilogue warpgroups: thread = token row t, warpgroup = column half
+        const int t = tid & 127;
+        const int half = warp >> 2;
+        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(a.y);
+        constexpr float kLog2e = 1.4426950408889634f;
+        for (int b = 0; b < nblk; ++b) {
+            const float *sc = scal + (b & 1) * kScFloats;
+            mbar_wait(&bars.sc_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            mbar_wait(&bars.ac_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            // G' row t, columns i = 64*half .. 64*half+63 -> K-block `half` of the operand in the C buffer
+            {
+                unsigned char *gk = sm + (b & 1) * kStageBytes + kXTile + kBTile + half * (kQ * 128);
+                const float lt = sc[t] * kLog2e;
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    uint32_t rr[32];
+                    tmem_ld32(lane_base + kTmG + 64 * half + 32 * q, rr);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float v[2];
+#pragma unroll
+                            for (int z = 0; z < 2; ++z) {
+                                const int il = 32 * q + 8 * c8 + 2 * e + z;
+                                const int i = 64 * half + il;
+                                // the exponent is a difference <= 0 for i <= t, so nothing can overflow
+                                const float dec = exp2f(lt - sc[i] * kLog2e);
+                                v[z] = (i <= t) ? __uint_as_float(rr[8 * c8 + 2 * e + z]) * dec * sc[3 * kQ + i] : 0.f;
+                            }
+                            w[e] = pack_bf16(v[0], v[1]);
+                        }
+                        *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 4 * q + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+            fence_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars.mg_ready);
+            // y_t[p] = Yintra + e^{l_t} Yinter, p = 32*half .. 32*half+31
+            mbar_wait(&bars.y_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            {
+                uint32_t ya[32], ye[32];
+                tmem_ld32(lane_base + kTmYa + 64 * (b & 1) + 32 * half, ya);
+                tmem_ld32(lane_base + kTmYe + 64 * (b & 1) + 32 * half, ye);
+                tmem_ld_wait();
+                const float et = sc[kQ + t];
+                const int tok = t_begin + b * kQ + t;
+                if (tok < t_end) {
+                    __nv_bfloat16 *dst = y + (static_cast<size_t>(tok) * a.H + h) * kP + 32 * half;
+#pragma unroll
+                    for (int c8 = 0; c8 < 4; ++c8) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int c = 8 * c8 + 2 * e;
+                            w[e] = pack_bf16(__uint_as_float(ya[c]) + et * __uint_as_float(ye[c]),
+                                             __uint_as_float(ya[c + 1]) + et * __uint_as_float(ye[c + 1]));
+                        }
+                        *reinterpret_cast<uint4 *>(dst + 8 * c8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars.yo_done[b & 1]);
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 13) tmem_dealloc(tm, kTmemCols);
+}
+
+}  // namespace
+
+bool ssd_scan_tensor_supported(const SsdArgs &a, bool io_bf16) {
+    return io_bf16 && a.P == kP && a.N == kN;
+}
+
+cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s) {
+    CUtensorMap mapX, mapB, mapC;
+    const uint64_t rows = static_cast<uint64_t>(a.T_total);
+    const uint64_t x_inner = static_cast<uint64_t>(a.H) * kP, bc_inner = static_cast<uint64_t>(a.G) * kN;
+    if (!make_tensor_map_2d(&mapX, a.x, 2, x_inner, rows, x_inner * 2, 64, kQ, true) ||
+        !make_tensor_map_2d(&mapB, a.B, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
+        !make_tensor_map_2d(&mapC, a.C, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(ssd_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    ssd_scan_tensor_kernel<<<dim3(a.H, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapX, mapB, mapC);
+    return cudaGetLastError();
+}
+
 }  // namespace lkv
