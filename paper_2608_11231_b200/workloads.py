@@ -32,9 +32,9 @@ CONFIGS = {
 def bf16_round(a) -> np.ndarray:
     """Round to the nearest bfloat16 (ties to even); result is float32."""
     x = np.ascontiguousarray(a, dtype=np.float32)
-    u = x.view(np.uint32).astype(np.uint64)
-    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(x.shape)
+    u = x.view(np.uint32)
+    u = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return u.view(np.float32).reshape(x.shape)
 
 
 def _io_round(a, io: str) -> np.ndarray:
@@ -59,9 +59,9 @@ def gdn_tokens(rng, T, H_k, H_v, d_k, d_v, io="bf16", live_chunk_len=None):
     (g * 4 / L, beta / 8) in which states carried across a cache chunk of L
     tokens stay well inside fp32 range, so that composition is observable.
     """
-    q = rng.standard_normal((T, H_k, d_k))
-    k = rng.standard_normal((T, H_k, d_k))
-    v = rng.standard_normal((T, H_v, d_v))
+    q = rng.standard_normal((T, H_k, d_k), dtype=np.float32)
+    k = rng.standard_normal((T, H_k, d_k), dtype=np.float32)
+    v = rng.standard_normal((T, H_v, d_v), dtype=np.float32)
     b_logit = rng.standard_normal((T, H_v))
     g_logit = rng.standard_normal((T, H_v))
     q /= np.linalg.norm(q, axis=-1, keepdims=True)
@@ -91,10 +91,10 @@ def ssd_tokens(rng, T, H, P, N, G, io="bf16"):
     x ~ N(0,1); dt = softplus(N(-2, sd 0.5)) (already activated);
     B, C ~ N(0,1) / sqrt(N).
     """
-    x = rng.standard_normal((T, H, P))
+    x = rng.standard_normal((T, H, P), dtype=np.float32)
     dt = _softplus(-2.0 + 0.5 * rng.standard_normal((T, H)))
-    B = rng.standard_normal((T, G, N)) / np.sqrt(N)
-    C = rng.standard_normal((T, G, N)) / np.sqrt(N)
+    B = rng.standard_normal((T, G, N), dtype=np.float32) / np.float32(np.sqrt(N))
+    C = rng.standard_normal((T, G, N), dtype=np.float32) / np.float32(np.sqrt(N))
     return dict(x=_io_round(x, io), dt=np.ascontiguousarray(dt, dtype=np.float32),
                 B=_io_round(B, io), C=_io_round(C, io))
 
