@@ -41,16 +41,9 @@ SSD_BLOCK = 128   # scan block of the tensor-core SSD kernel (tokens)
 # ----------------------------------------------------------------------------- workload description
 
 def build_requests(name: str, rank: int = 0):
-    """List of requests: family, number of cached chunks K, context tokens, recompute tokens."""
-    if name == "cfg1":
-        return [dict(family="mamba2", K=8, total=8 * 1024, recompute=1024)]
-    if name == "cfg2":
-        return [dict(family="gdn", K=16, total=16 * 1024, recompute=int(0.2 * 16 * 1024))]
-    if name == "cfg3":
-        return [dict(family="gdn", K=32, total=32 * 1024, recompute=2048, shared_pool=True) for _ in range(8)]
-    if name == "cfg4":
-        return wl.ragged_mix(seed=4 + 1000 * rank)
-    raise ValueError(name)
+    """List of requests of this rank: family, number of cached chunks K, context tokens, recompute tokens."""
+    from paper_2608_11231_b200 import sharding
+    return sharding.rank_requests(name, rank)
 
 
 def gdn_scan_flops(tokens: int, s=GDN_SHAPE, C=GDN_BLOCK) -> float:
@@ -276,6 +269,8 @@ def run_ours(args):
     torch.cuda.synchronize()
     context_tokens = sum(f.context_tokens for f in fams)
     scan_tokens = sum(f.scan_tokens for f in fams)
+    job_context_tokens = context_tokens
+    job_scan_tokens = scan_tokens
 
     def barrier():
         torch.cuda.synchronize()
@@ -283,12 +278,10 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    from paper_2608_11231_b200 import sharding
+
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.job_step_ms(x, dist if world > 1 else None, "cuda")
 
     total_input_bytes = sum(f.h2d_bytes for f in fams)
     cold_by_size = total_input_bytes > 4 * 126e6        # inputs far larger than the 126 MB L2
@@ -370,6 +363,9 @@ def run_ours(args):
     step_e2e()
     ms_e2e = timed_back_to_back(step_e2e, e2e_steps)
 
+    if world > 1:
+        job_context_tokens = sharding.job_total(context_tokens, dist, "cuda")
+        job_scan_tokens = sharding.job_total(scan_tokens, dist, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -415,18 +411,18 @@ def run_ours(args):
 
     base, _ = cpu_baseline_sample() if world == 1 else (None, None)
     line = dict(
-        metric=METRIC, value=world * context_tokens / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
+        metric=METRIC, value=job_context_tokens / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
         warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="bf16", data="synthetic",
         config=dict(workload=args.workload, requests=len(reqs), context_tokens=context_tokens,
                     scan_tokens=scan_tokens, l2="inputs far larger than L2, steps timed back to back" if cold_by_size else
                     "L2 flushed (512 MiB write, untimed) before every timed step", timing="CUDA-graph replay, CUDA events",
                     sharding="requests across ranks, no collective"),
-        e2e=dict(value=world * context_tokens / (ms_e2e * 1e-3), unit=UNIT,
+        e2e=dict(value=job_context_tokens / (ms_e2e * 1e-3), unit=UNIT,
                  h2d_bytes_per_step=sum(f.h2d_bytes for f in fams), d2h_bytes_per_step=sum(f.d2h_bytes for f in fams),
                  ms_per_step=ms_e2e, steps=e2e_steps),
         gpu_launches=sum(f.launches for f in fams) * args.steps,
-        scan_tokens_per_s=world * scan_tokens / (ms * 1e-3),
+        scan_tokens_per_s=job_scan_tokens / (ms * 1e-3),
         roofline=roof, kernels=detail, clocks=clocks)
     if base is not None:
         line["cpu_baseline"] = base

@@ -42,9 +42,10 @@ constexpr int kOffR = kOffSt + 2 * kD * 128;           // R^T bf16 [128 rows x 1
 constexpr int kOffUw = kOffR + kD * 128;               // (U o w)^T bf16
 constexpr int kOffMPM = kOffUw + kD * 128;             // [M; PM] bf16 [128 rows x 128 B], double-buffered
 constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] (A operand of (6); rows 64..127 unused)
+constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
 constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i]
-constexpr int kOffM = kOffA + kC * kC * 4;             // M fp32 [t][i]
-constexpr int kOffT = kOffM + kC * kC * 4;             // block-product scratch, 3 x 16 x 16 fp32
+constexpr int kOffM = kOffA + kC * kLd * 4;            // M fp32 [t][i]
+constexpr int kOffT = kOffM + kC * kLd * 4;            // block-product scratch, 3 x 16 x 16 fp32
 constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, double-buffered
 constexpr int kGbFloats = 4 * kC;                      // cg, beta, gam (e^{cg}), w (e^{cg_C - cg})
 constexpr int kSmemBytes = kOffGb + 2 * kGbFloats * 4 + 1024;
@@ -76,10 +77,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
-// 32 consecutive fp32 values -> bf16, written as 4 swizzled 16-byte chunks (chunk0 .. chunk0+3) of operand row `row`
-__device__ __forceinline__ void store_row_chunks(unsigned char *tile, int row, int chunk0, const float (&v)[32]) {
+// 16 consecutive fp32 values -> bf16, written as 2 swizzled 16-byte chunks (chunk0, chunk0+1) of operand row `row`
+__device__ __forceinline__ void store_row_chunks(unsigned char *tile, int row, int chunk0, const float (&v)[16]) {
 #pragma unroll
-    for (int c8 = 0; c8 < 4; ++c8) {
+    for (int c8 = 0; c8 < 2; ++c8) {
         uint32_t w[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) w[e] = pack_bf16(v[8 * c8 + 2 * e], v[8 * c8 + 2 * e + 1]);
@@ -268,28 +269,28 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             {
                 const int t = x & 63;
                 const float cgt = sc[t], bt = sc[kC + t];
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t rr[32];
-                    tmem_ld32(lane_base + kTmG + 32 * q, rr);
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t rr[16];
+                    tmem_ld16(lane_base + kTmG + 16 * q, rr);
                     tmem_ld_wait();
-                    float v[32];
+                    float v[16];
                     if (x < kC) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int i = 32 * q + c;
+                        for (int c = 0; c < 16; ++c) {
+                            const int i = 16 * q + c;
                             v[c] = (i <= t) ? __expf(cgt - sc[i]) * __uint_as_float(rr[c]) : 0.f;
                         }
-                        store_row_chunks(sm + kOffP, t, 4 * q, v);
+                        store_row_chunks(sm + kOffP, t, 2 * q, v);
                     } else {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int i = 32 * q + c;
+                        for (int c = 0; c < 16; ++c) {
+                            const int i = 16 * q + c;
                             v[c] = (i < t) ? bt * __expf(cgt - sc[i]) * __uint_as_float(rr[c]) : 0.f;
                         }
 #pragma unroll
-                        for (int c = 0; c < 32; c += 4)
-                            *reinterpret_cast<float4 *>(Af + t * kC + 32 * q + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                        for (int c = 0; c < 16; c += 4)
+                            *reinterpret_cast<float4 *>(Af + t * kLd + 16 * q + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
                     }
                 }
             }
@@ -298,17 +299,17 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k.
             if (x < kC) {
                 const int k = x >> 4, c = x & 15;
-                const float *Ab = Af + (16 * k) * kC + 16 * k;
+                const float *Ab = Af + (16 * k) * kLd + 16 * k;
                 float xv[16];
 #pragma unroll
                 for (int t = 0; t < 16; ++t) {
                     float acc = (t == c) ? 1.f : 0.f;
 #pragma unroll
-                    for (int i = 0; i < t; ++i) acc = fmaf(-Ab[t * kC + i], xv[i], acc);
+                    for (int i = 0; i < t; ++i) acc = fmaf(-Ab[t * kLd + i], xv[i], acc);
                     xv[t] = (t >= c) ? acc : 0.f;
                 }
 #pragma unroll
-                for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kC + 16 * k + c] = xv[t];
+                for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
             }
             named_bar_sync(1, 128);
             // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc.
@@ -317,11 +318,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 const int nstrip = (4 - d) * 64;
                 for (int e = x; e < nstrip; e += 128) {
                     const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *arow = Af + (16 * r + tt) * kC;
+                    const float *arow = Af + (16 * r + tt) * kLd;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int ii = 16 * c; ii < 16 * r; ++ii) {
                         const float av = arow[ii];
-                        const float4 mv = *reinterpret_cast<const float4 *>(Mf + ii * kC + 16 * c + 4 * lg);
+                        const float4 mv = *reinterpret_cast<const float4 *>(Mf + ii * kLd + 16 * c + 4 * lg);
                         acc.x = fmaf(av, mv.x, acc.x); acc.y = fmaf(av, mv.y, acc.y);
                         acc.z = fmaf(av, mv.z, acc.z); acc.w = fmaf(av, mv.w, acc.w);
                     }
@@ -330,7 +331,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 named_bar_sync(1, 128);
                 for (int e = x; e < nstrip; e += 128) {
                     const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *drow = Mf + (16 * r + tt) * kC + 16 * r;
+                    const float *drow = Mf + (16 * r + tt) * kLd + 16 * r;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
                     for (int i = 0; i < 16; ++i) {
@@ -339,7 +340,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                         acc.x = fmaf(dv, tv.x, acc.x); acc.y = fmaf(dv, tv.y, acc.y);
                         acc.z = fmaf(dv, tv.z, acc.z); acc.w = fmaf(dv, tv.w, acc.w);
                     }
-                    *reinterpret_cast<float4 *>(Mf + (16 * r + tt) * kC + 16 * c + 4 * lg) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
+                    *reinterpret_cast<float4 *>(Mf + (16 * r + tt) * kLd + 16 * c + 4 * lg) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
                 }
                 named_bar_sync(1, 128);
             }
@@ -347,16 +348,16 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
             if (x < kC) {
                 const int t = x;
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    float v[16];
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    float v[32];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const int i = 32 * q + c;
-                        const float4 mv = (i >> 4) <= (t >> 4) ? *reinterpret_cast<const float4 *>(Mf + t * kC + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int c = 0; c < 16; c += 4) {
+                        const int i = 16 * q + c;
+                        const float4 mv = (i >> 4) <= (t >> 4) ? *reinterpret_cast<const float4 *>(Mf + t * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
                         v[c] = mv.x; v[c + 1] = mv.y; v[c + 2] = mv.z; v[c + 3] = mv.w;
                     }
-                    store_row_chunks(mpm, t, 4 * q, v);
+                    store_row_chunks(mpm, t, 2 * q, v);
                 }
             }
             fence_async_smem();
@@ -365,15 +366,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
             if (x < kC) {
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t rr[32];
-                    tmem_ld32(lane_base + kTmG + 32 * q, rr);
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t rr[16];
+                    tmem_ld16(lane_base + kTmG + 16 * q, rr);
                     tmem_ld_wait();
-                    float v[32];
+                    float v[16];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(rr[c]);
-                    store_row_chunks(mpm, kC + x, 4 * q, v);
+                    for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
+                    store_row_chunks(mpm, kC + x, 2 * q, v);
                 }
             }
             fence_async_smem();
@@ -395,15 +396,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const int t0 = t_begin + b * kC;
             const int n = min(kC, t_end - t0);
             __nv_bfloat16 *orow = o + (static_cast<size_t>(t0) * a.H_v + h) * kD + j;
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                uint32_t qs[32], pu[32];
-                tmem_ld32(lane_base + kTmD1 + 32 * q, qs);
-                tmem_ld32(lane_base + kTmUP + kC + 32 * q, pu);
+#pragma unroll 1
+            for (int q = 0; q < 8; ++q) {
+                uint32_t qs[8], pu[8];
+                tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
+                tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
                 tmem_ld_wait();
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const int t = 32 * q + c;
+                for (int c = 0; c < 8; ++c) {
+                    const int t = 8 * q + c;
                     const float val = a.scale * fmaf(sc[2 * kC + t], __uint_as_float(qs[c]), __uint_as_float(pu[c]));
                     if (t < n) orow[t * tstride] = __float2bfloat16_rn(val);
                 }
@@ -419,17 +420,17 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         mbar_wait(&bars.gb_ready[0], 0, &dead, a.status);
         {
             const float gamC = gb[2 * kC + kC - 1];
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                float v[16];
+                uint32_t rr[16];
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                float v[32];
-                uint32_t rr[32];
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    v[c] = a.S0 ? a.S0[sbase + static_cast<size_t>(64 * half + 32 * q + c) * kD + j] : 0.f;
+                for (int c = 0; c < 16; ++c) {
+                    v[c] = a.S0 ? a.S0[sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j] : 0.f;
                     rr[c] = __float_as_uint(v[c] * gamC);
                 }
-                tmem_st32(lane_base + kTmS + 64 * half + 32 * q, rr);
-                store_row_chunks(sm + kOffSt + half * (kD * 128), j, 4 * q, v);
+                tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);
+                store_row_chunks(sm + kOffSt + half * (kD * 128), j, 2 * q, v);
             }
             tmem_st_wait();
             fence_async_smem();
@@ -445,17 +446,18 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.d1_done, par, &dead, a.status);
             tc_fence_after_sync();
             // r_t = beta_t (v_t[j] - gam_t (S^T k_t)_j), t = 32*half..+31 -> R^T row j
-            {
-                uint32_t rr[32];
-                tmem_ld32(lane_base + kTmD1 + kC + 32 * half, rr);
+#pragma unroll 1
+            for (int q = 0; q < 2; ++q) {
+                uint32_t rr[16];
+                tmem_ld16(lane_base + kTmD1 + kC + 32 * half + 16 * q, rr);
                 tmem_ld_wait();
-                float v[32];
+                float v[16];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const int t = 32 * half + c;
+                for (int c = 0; c < 16; ++c) {
+                    const int t = 32 * half + 16 * q + c;
                     v[c] = sc[kC + t] * (__bfloat162float(vt[t * kD + j]) - sc[2 * kC + t] * __uint_as_float(rr[c]));
                 }
-                store_row_chunks(sm + kOffR, j, 4 * half, v);
+                store_row_chunks(sm + kOffR, j, 4 * half + 2 * q, v);
             }
             mbar_arrive(&bars.v_free);
             fence_async_smem();
@@ -464,14 +466,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             // (U o w)^T row j, i = 32*half..+31
             mbar_wait(&bars.up_done, par, &dead, a.status);
             tc_fence_after_sync();
-            {
-                uint32_t rr[32];
-                tmem_ld32(lane_base + kTmUP + 32 * half, rr);
+#pragma unroll 1
+            for (int q = 0; q < 2; ++q) {
+                uint32_t rr[16];
+                tmem_ld16(lane_base + kTmUP + 32 * half + 16 * q, rr);
                 tmem_ld_wait();
-                float v[32];
+                float v[16];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) v[c] = __uint_as_float(rr[c]) * sc[3 * kC + 32 * half + c];
-                store_row_chunks(sm + kOffUw, j, 4 * half, v);
+                for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]) * sc[3 * kC + 32 * half + 16 * q + c];
+                store_row_chunks(sm + kOffUw, j, 4 * half + 2 * q, v);
             }
             fence_async_smem();
             tc_fence_before_sync();
@@ -485,26 +488,26 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 mbar_wait(&bars.gb_ready[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
                 gamN = gb[((b + 1) & 1) * kGbFloats + 2 * kC + kC - 1];
             }
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                uint32_t rr[32];
-                tmem_ld32(lane_base + kTmS + 64 * half + 32 * q, rr);
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                uint32_t rr[16];
+                tmem_ld16(lane_base + kTmS + 64 * half + 16 * q, rr);
                 tmem_ld_wait();
                 if (last) {
                     if (a.S_T) {
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            a.S_T[sbase + static_cast<size_t>(64 * half + 32 * q + c) * kD + j] = __uint_as_float(rr[c]);
+                        for (int c = 0; c < 16; ++c)
+                            a.S_T[sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j] = __uint_as_float(rr[c]);
                     }
                 } else {
-                    float v[32];
+                    float v[16];
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
+                    for (int c = 0; c < 16; ++c) {
                         v[c] = __uint_as_float(rr[c]);
                         rr[c] = __float_as_uint(v[c] * gamN);
                     }
-                    tmem_st32(lane_base + kTmS + 64 * half + 32 * q, rr);
-                    store_row_chunks(sm + kOffSt + half * (kD * 128), j, 4 * q, v);
+                    tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);
+                    store_row_chunks(sm + kOffSt + half * (kD * 128), j, 2 * q, v);
                 }
             }
             if (!last) {
