@@ -47,7 +47,9 @@ constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i]
 constexpr int kOffM = kOffA + kC * kLd * 4;            // M fp32 [t][i]
 constexpr int kOffT = kOffM + kC * kLd * 4;            // block-product scratch, 3 x 16 x 16 fp32
 constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, double-buffered
-constexpr int kGbFloats = 4 * kC;                      // cg, beta, gam (e^{cg}), w (e^{cg_C - cg})
+constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kMaxGroupRange = 100.f;                // log2 units: above this the per-group factors could overflow
 constexpr int kSmemBytes = kOffGb + 2 * kGbFloats * 4 + 1024;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
@@ -257,9 +259,18 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 if (x == 31) scan_carry = run;
                 named_bar_sync(1, 128);
                 if (x >= 32 && x < kC) run += scan_carry;
-                if (x < kC) { sc[x] = run; sc[kC + x] = bv; sc[2 * kC + x] = __expf(run); }
+                const float c2 = run * kLog2e;
+                if (x < kC) { sc[x] = c2; sc[kC + x] = bv; sc[2 * kC + x] = exp2f(c2); }
                 named_bar_sync(1, 128);
-                if (x < kC) sc[3 * kC + x] = __expf(sc[kC - 1] - run);
+                if (x < kC) {
+                    sc[3 * kC + x] = exp2f(sc[kC - 1] - c2);
+                    // factor of column x relative to the first column of its group of 16 (>= 1)
+                    const float rng = sc[x & ~15] - c2;
+                    sc[4 * kC + x] = exp2f(fminf(rng, 126.f));
+                    const unsigned bad = __ballot_sync(0xffffffffu, rng > kMaxGroupRange);
+                    if (x == 0) sc[5 * kC] = bad ? 1.f : 0.f;
+                    if (x == 32) sc[5 * kC + 1] = bad ? 1.f : 0.f;
+                }
                 named_bar_sync(1, 128);
                 mbar_arrive(&bars.gb_ready[b & 1]);
             }
@@ -267,27 +278,40 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.g_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
             {
+                // Gam_ti = 2^{cg2_t - cg2_ref} * f_i with ref the first column of i's group of 16: one exponential
+                // per group (both factors' product is <= 1 where i <= t); violent decay takes the per-element path
                 const int t = x & 63;
-                const float cgt = sc[t], bt = sc[kC + t];
+                const float cgt = sc[t];
+                const float coef = (x < kC) ? 1.f : sc[kC + t];     // rows of P: 1, rows of A: beta_t
+                const int lim = (x < kC) ? t : t - 1;               // P keeps the diagonal, A is strictly lower
+                const bool fast = sc[5 * kC] + sc[5 * kC + 1] == 0.f;
 #pragma unroll 1
                 for (int q = 0; q < 4; ++q) {
                     uint32_t rr[16];
                     tmem_ld16(lane_base + kTmG + 16 * q, rr);
                     tmem_ld_wait();
+                    const int i0 = 16 * q;
                     float v[16];
-                    if (x < kC) {
+                    if (fast) {
+                        float aa;
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(cgt - sc[i0], 0.f)));
+                        aa *= coef;
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int i = 16 * q + c;
-                            v[c] = (i <= t) ? __expf(cgt - sc[i]) * __uint_as_float(rr[c]) : 0.f;
+                        for (int c = 0; c < 16; c += 4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                            v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                            v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                            v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                            v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
                         }
-                        store_row_chunks(sm + kOffP, t, 2 * q, v);
                     } else {
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int i = 16 * q + c;
-                            v[c] = (i < t) ? bt * __expf(cgt - sc[i]) * __uint_as_float(rr[c]) : 0.f;
-                        }
+                        for (int c = 0; c < 16; ++c)
+                            v[c] = (i0 + c <= lim) ? coef * exp2f(cgt - sc[i0 + c]) * __uint_as_float(rr[c]) : 0.f;
+                    }
+                    if (x < kC) {
+                        store_row_chunks(sm + kOffP, t, 2 * q, v);
+                    } else {
 #pragma unroll
                         for (int c = 0; c < 16; c += 4)
                             *reinterpret_cast<float4 *>(Af + t * kLd + 16 * q + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);

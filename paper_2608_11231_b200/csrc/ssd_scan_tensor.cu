@@ -36,7 +36,9 @@ constexpr int kStageBytes = kXTile + kBTile + kCTile;   // 80 KB
 constexpr int kOffX2 = 2 * kStageBytes;     // X~ [128 tokens x 64 p]
 constexpr int kOffHb = kOffX2 + kXTile;     // bf16 state [128 n x 64 p]
 constexpr int kOffSc = kOffHb + kN * 128;   // per-block scalars, double-buffered
-constexpr int kScFloats = 4 * kQ;           // l, e^{l}, s = e^{l_Q - l} dt, dt
+constexpr int kScFloats = 5 * kQ + 4;       // l2 = l log2(e), e^{l}, s = e^{l_Q - l} dt, f = e^{l_ref - l} dt, dt, flag
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kMaxGroupRange = 100.f;     // log2 units: above this the per-group factors could overflow
 constexpr int kSmemBytes = kOffSc + 2 * kScFloats * 4 + 1024;
 
 // tensor-memory map (columns)
@@ -187,11 +189,20 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             if (lane == 31) scan_carry[warp & 3] = run;
             named_bar_sync(1, 128);
             for (int w = 0; w < (warp & 3); ++w) run += scan_carry[w];
-            dst[x] = run;
-            dst[kQ + x] = __expf(run);
+            const float l2 = run * kLog2e;
+            dst[x] = l2;
+            dst[kQ + x] = exp2f(l2);
+            dst[4 * kQ + x] = dtv;
             named_bar_sync(1, 128);
-            dst[2 * kQ + x] = __expf(dst[kQ - 1] - run) * dtv;
-            dst[3 * kQ + x] = dtv;
+            dst[2 * kQ + x] = exp2f(dst[kQ - 1] - l2) * dtv;
+            // factor of column x relative to the first column of its group of 16 (>= 1 before dt)
+            const float rng = dst[x & ~15] - l2;
+            dst[3 * kQ + x] = exp2f(fminf(rng, 126.f)) * dtv;
+            // the fast epilogue is exact only while no group spans more than kMaxGroupRange
+            const unsigned bad = __ballot_sync(0xffffffffu, rng > kMaxGroupRange);
+            if (lane == 0) scan_carry[warp & 3] = bad ? 1.f : 0.f;
+            named_bar_sync(1, 128);
+            if (x == 0) dst[5 * kQ] = scan_carry[0] + scan_carry[1] + scan_carry[2] + scan_carry[3];
             named_bar_sync(1, 128);
             mbar_arrive(&bars.sc_ready[b & 1]);
         };
@@ -291,39 +302,49 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
         const int half = warp >> 2;
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(a.y);
-        constexpr float kLog2e = 1.4426950408889634f;
         for (int b = 0; b < nblk; ++b) {
             const float *sc = scal + (b & 1) * kScFloats;
             mbar_wait(&bars.sc_ready[b & 1], (b >> 1) & 1, &dead, a.status);
             mbar_wait(&bars.ac_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
-            // G' row t, columns i = 64*half .. 64*half+63 -> K-block `half` of the operand in the C buffer
+            // G' row t, columns i = 64*half .. 64*half+63 -> K-block `half` of the operand in the C buffer.
+            // e^{l_t - l_i} dt_i = 2^{l2_t - l2_ref} * f_i with ref the first column of i's group of 16: one
+            // exponential per group instead of one per element (every factor is <= 1 where i <= t);
+            // blocks whose decay is too violent for that take the per-element path.
             {
                 unsigned char *gk = sm + (b & 1) * kStageBytes + kXTile + kBTile + half * (kQ * 128);
-                const float lt = sc[t] * kLog2e;
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    uint32_t rr[32];
-                    tmem_ld32(lane_base + kTmG + 64 * half + 32 * q, rr);
+                const float lt = sc[t];
+                const bool fast = sc[5 * kQ] == 0.f;
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t rr[16];
+                    tmem_ld16(lane_base + kTmG + 64 * half + 16 * q, rr);
                     tmem_ld_wait();
+                    const int i0 = 64 * half + 16 * q;
+                    uint32_t w[8];
+                    if (fast) {
+                        float aa;
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(lt - sc[i0], 0.f)));
 #pragma unroll
-                    for (int c8 = 0; c8 < 4; ++c8) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            float v[2];
-#pragma unroll
-                            for (int z = 0; z < 2; ++z) {
-                                const int il = 32 * q + 8 * c8 + 2 * e + z;
-                                const int i = 64 * half + il;
-                                // the exponent is a difference <= 0 for i <= t, so nothing can overflow
-                                const float dec = exp2f(lt - sc[i] * kLog2e);
-                                v[z] = (i <= t) ? __uint_as_float(rr[8 * c8 + 2 * e + z]) * dec * sc[3 * kQ + i] : 0.f;
-                            }
-                            w[e] = pack_bf16(v[0], v[1]);
+                        for (int c = 0; c < 16; c += 4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(sc + 3 * kQ + i0 + c);
+                            const float v0 = (i0 + c <= t) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                            const float v1 = (i0 + c + 1 <= t) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                            const float v2 = (i0 + c + 2 <= t) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                            const float v3 = (i0 + c + 3 <= t) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                            w[c / 2] = pack_bf16(v0, v1);
+                            w[c / 2 + 1] = pack_bf16(v2, v3);
                         }
-                        *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 4 * q + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; c += 2) {
+                            const float v0 = (i0 + c <= t) ? __uint_as_float(rr[c]) * exp2f(lt - sc[i0 + c]) * sc[4 * kQ + i0 + c] : 0.f;
+                            const float v1 = (i0 + c + 1 <= t) ? __uint_as_float(rr[c + 1]) * exp2f(lt - sc[i0 + c + 1]) * sc[4 * kQ + i0 + c + 1] : 0.f;
+                            w[c / 2] = pack_bf16(v0, v1);
+                        }
                     }
+                    *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 2 * q)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 2 * q + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
                 }
             }
             fence_async_smem();

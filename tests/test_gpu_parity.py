@@ -376,3 +376,25 @@ def test_gdn_exact_tensor_many_heads_ragged():
         assert maxrel(got[r], ref) <= 2e-3, (r, k, maxrel(got[r], ref))
     assert got[1].tobytes() == pool[ids[cu[1]]].tobytes()
     assert not got[2].any()
+
+
+def test_scans_with_violent_decay_take_the_exact_exponent_path():
+    """Decay so strong that a 16-token group spans more than 2^100: the tensor-core kernels must fall back to
+    per-element exponents (the grouped form would overflow) and still match the token recurrence."""
+    torch = _torch()
+    bf = torch.bfloat16
+    rng = np.random.default_rng(77)
+    tok = wl.gdn_tokens(rng, 200, 2, 4, 128, 128)
+    tok["g"] = (tok["g"] * 80.0).astype(np.float32)            # about -6 per token
+    assert (tok["g"].min() * 16 * 1.4427) < -100
+    S0 = rng.standard_normal((1, 4, 128, 128)).astype(np.float32)
+    o, ST = _run_gdn(tok, S0, "bf16")
+    o_ref, ST_ref = oracle.gdn_seq(tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], S0[0])
+    assert maxrel(o, o_ref) <= TOL_BF16 and maxrel(ST[0], ST_ref) <= TOL_BF16
+    H, P, N, G = 4, 64, 128, 1
+    A = (wl.ssd_A(rng, H) * 12.0).astype(np.float32)          # dt * A about -6 per token and more
+    st = wl.ssd_tokens(rng, 300, H, P, N, G)
+    assert (st["dt"].max() * A.min() * 16 * 1.4427) < -100
+    y, hT = _run_ssd(st, A, rng.standard_normal((1, H, N, P)).astype(np.float32) * 0 + 1.0, "bf16")
+    y_ref, hT_ref = oracle.ssd_seq(st["x"], st["dt"], A, st["B"], st["C"], np.ones((H, N, P)))
+    assert maxrel(y, y_ref) <= TOL_BF16 and maxrel(hT[0], hT_ref) <= TOL_BF16
