@@ -39,12 +39,12 @@ constexpr int kQKStage = 4 * kC * 128;                 // [Q_kb0 | K_kb0 | Q_kb1
 constexpr int kOffV = 2 * kQKStage;                    // V tile [64][128] bf16, row-major (single buffer)
 constexpr int kOffSt = kOffV + kC * kD * 2;            // S^T bf16: [St_kb0 | St_kb1], each [128 rows x 128 B]
 constexpr int kOffR = kOffSt + 2 * kD * 128;           // R^T bf16 [128 rows x 128 B]
-constexpr int kOffUw = kOffR + kD * 128;               // (U o w)^T bf16
-constexpr int kOffMPM = kOffUw + kD * 128;             // [M; PM] bf16 [128 rows x 128 B], double-buffered
+constexpr int kOffUw = kOffR;                          // (U o w)^T bf16: written only after (3) has consumed R^T
+constexpr int kOffMPM = kOffR + kD * 128;              // [M; PM] bf16 [128 rows x 128 B], double-buffered
 constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] (A operand of (6); rows 64..127 unused)
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
-constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i]
-constexpr int kOffM = kOffA + kC * kLd * 4;            // M fp32 [t][i]
+constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
+constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
 constexpr int kOffT = kOffM + kC * kLd * 4;            // block-product scratch, 3 x 16 x 16 fp32
 constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, double-buffered
 constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
@@ -54,7 +54,8 @@ constexpr int kSmemBytes = kOffGb + 2 * kGbFloats * 4 + 1024;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 // tensor-memory map (columns)
-constexpr uint32_t kTmG = 0;      // 64: G, then PM
+constexpr uint32_t kTmG = 0;      // 64
+constexpr uint32_t kTmPM = 448;   // 64
 constexpr uint32_t kTmD1 = 64;    // 128: QS | KS
 constexpr uint32_t kTmUP = 192;   // 128: U | PU
 constexpr uint32_t kTmS = 320;    // 128
@@ -64,7 +65,9 @@ struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
     uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done;
     // 128-thread barriers (prep or out warpgroup)
-    uint64_t gb_ready[2], m_ready, mpm_ready[2], o_done[2];
+    uint64_t gb_ready[2], m_ready, mpm_ready[2], o_done[2], inv_done[2];
+    // 64-thread barriers (the two halves of the out warpgroup)
+    uint64_t a_ready, p_ready;
     // 256-thread barriers (both chain warpgroups)
     uint64_t v_free, r_ready, uw_ready, st_ready, chain_done[2];
 };
@@ -117,7 +120,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         uint64_t *b1 = &bars.full_qk[0];
         for (int i = 0; i < 10; ++i) mbar_init(b1 + i, 1);
         uint64_t *b128 = &bars.gb_ready[0];
-        for (int i = 0; i < 7; ++i) mbar_init(b128 + i, 128);
+        for (int i = 0; i < 9; ++i) mbar_init(b128 + i, 128);
+        mbar_init(&bars.a_ready, 64);
+        mbar_init(&bars.p_ready, 64);
         uint64_t *b256 = &bars.v_free;
         for (int i = 0; i < 6; ++i) mbar_init(b256 + i, 256);
         mbar_fence_init();
@@ -174,13 +179,14 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             auto issue_PM = [&](int b) {   // PM = P M: A = P (K = i), B = M rows of the [M; PM] tile read MN-major
                 const uint64_t dM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmG, dP + 2 * k, dM + ((k * 16 * 128) >> 4), idPM, k > 0);
+                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmPM, dP + 2 * k, dM + ((k * 16 * 128) >> 4), idPM, k > 0);
                 umma_commit(&bars.pm_done);
             };
             mbar_wait(&bars.full_qk[0], 0, &dead, a.status);
             tc_fence_after_sync();
             issue_G(0);
             mbar_wait(&bars.m_ready, 0, &dead, a.status);
+            mbar_wait(&bars.p_ready, 0, &dead, a.status);
             tc_fence_after_sync();
             issue_PM(0);
             for (int b = 0; b < nblk; ++b) {
@@ -197,15 +203,16 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
                 }
                 umma_commit(&bars.d1_done);
-                // [M; PM] of block b complete, which also means the G / PM columns are drained
-                mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
-                // (1) of the next block right behind (2): the prep warps then work while the chain runs block b
+                // (1) of the next block right behind (2), as soon as the epilogue of block b has drained the G columns
                 if (b + 1 < nblk) {
+                    mbar_wait(&bars.a_ready, par, &dead, a.status);
+                    mbar_wait(&bars.p_ready, par, &dead, a.status);
                     mbar_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
                     tc_fence_after_sync();
                     issue_G(b + 1);
                 }
                 // (3) [U | PU] = R^T [M; PM]^T
+                mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
                 mbar_wait(&bars.r_ready, par, &dead, a.status);
                 tc_fence_after_sync();
                 const uint64_t dMPM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
@@ -223,6 +230,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 // (6) of the next block once its inverse is ready
                 if (b + 1 < nblk) {
                     mbar_wait(&bars.m_ready, (b + 1) & 1, &dead, a.status);
+                    mbar_wait(&bars.p_ready, (b + 1) & 1, &dead, a.status);
                     tc_fence_after_sync();
                     issue_PM(b + 1);
                 }
@@ -232,9 +240,18 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         // ======================================================= prep warpgroup (one block ahead)
         const int x = tid - 384;                 // 0..127 = TMEM lane
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        float *Af = reinterpret_cast<float *>(sm + kOffA);
         float *Mf = reinterpret_cast<float *>(sm + kOffM);
         float *Tt = reinterpret_cast<float *>(sm + kOffT);
+        auto fetch_gb = [&](int b, float &gv, float &bv) {
+            const int t = t_begin + b * kC + x;
+            gv = 0.f; bv = 0.f;
+            if (x < kC && b < nblk && t < t_end) {
+                gv = a.g[static_cast<size_t>(t) * a.H_v + h];
+                bv = a.beta[static_cast<size_t>(t) * a.H_v + h];
+            }
+        };
+        float gv_next, bv_next;
+        fetch_gb(0, gv_next, bv_next);
         for (int b = 0; b < nblk; ++b) {
             // buffers of parity b were last used by block b-2
             if (b >= 2) {
@@ -244,12 +261,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             // ---- per-block scalars: cg, beta, gam = e^{cg}, w = e^{cg_C - cg}
             float *sc = gb + (b & 1) * kGbFloats;
             {
-                const int t0 = t_begin + b * kC;
-                float gv = 0.f, bv = 0.f;
-                if (x < kC && t0 + x < t_end) {
-                    gv = a.g[static_cast<size_t>(t0 + x) * a.H_v + h];
-                    bv = a.beta[static_cast<size_t>(t0 + x) * a.H_v + h];
-                }
+                const float gv = gv_next, bv = bv_next;
+                fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
                 float run = gv;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
@@ -274,7 +287,144 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 named_bar_sync(1, 128);
                 mbar_arrive(&bars.gb_ready[b & 1]);
             }
-            // ---- epilogue of (1): rows 0..63 -> P (bf16 operand), rows 64..127 -> A (fp32)
+            // ---- P and A come from the out warpgroup (epilogue of (1))
+            mbar_wait(&bars.a_ready, b & 1, &dead, a.status);
+            const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
+            // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k by forward
+            // substitution; each row of the block is fetched with four 16-byte loads ahead of its use.
+            if (x < kC) {
+                const int k = x >> 4, c = x & 15;
+                const float *Ab = Af + (16 * k) * kLd + 16 * k;
+                float xv[16];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) {
+                    float row[16];
+#pragma unroll
+                    for (int i4 = 0; i4 < 16; i4 += 4) {
+                        if (i4 < t) {
+                            const float4 v = *reinterpret_cast<const float4 *>(Ab + t * kLd + i4);
+                            row[i4] = v.x; row[i4 + 1] = v.y; row[i4 + 2] = v.z; row[i4 + 3] = v.w;
+                        }
+                    }
+                    float acc0 = (t == c) ? 1.f : 0.f, acc1 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < t; ++i) {
+                        if (i & 1) acc1 = fmaf(-row[i], xv[i], acc1);
+                        else acc0 = fmaf(-row[i], xv[i], acc0);
+                    }
+                    xv[t] = (t >= c) ? acc0 + acc1 : 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
+            }
+            named_bar_sync(1, 128);
+            // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc.
+            // A thread owns a 1 x 4 strip (row tt, columns 4*lg..4*lg+3) of a 16 x 16 block; operands are fetched
+            // eight k-steps at a time with 16-byte loads so that the loads of a group are in flight together.
+            for (int d = 1; d < 4; ++d) {
+                const int nstrip = (4 - d) * 64;
+                for (int e = x; e < nstrip; e += 128) {
+                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
+                    const float *arow = Af + (16 * r + tt) * kLd;
+                    const float *mcol = Mf + 16 * c + 4 * lg;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+                    for (int ii = 16 * c; ii < 16 * r; ii += 8) {
+                        const float4 a0 = *reinterpret_cast<const float4 *>(arow + ii);
+                        const float4 a1 = *reinterpret_cast<const float4 *>(arow + ii + 4);
+                        float4 mv[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) mv[u] = *reinterpret_cast<const float4 *>(mcol + (ii + u) * kLd);
+                        const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            acc.x = fmaf(av[u], mv[u].x, acc.x); acc.y = fmaf(av[u], mv[u].y, acc.y);
+                            acc.z = fmaf(av[u], mv[u].z, acc.z); acc.w = fmaf(av[u], mv[u].w, acc.w);
+                        }
+                    }
+                    *reinterpret_cast<float4 *>(Tt + c * 256 + tt * 16 + 4 * lg) = acc;
+                }
+                named_bar_sync(1, 128);
+                for (int e = x; e < nstrip; e += 128) {
+                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
+                    const float *drow = Mf + (16 * r + tt) * kLd + 16 * r;
+                    const float *tcol = Tt + c * 256 + 4 * lg;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int i = 0; i < 16; i += 8) {
+                        const float4 d0 = *reinterpret_cast<const float4 *>(drow + i);
+                        const float4 d1 = *reinterpret_cast<const float4 *>(drow + i + 4);
+                        float4 tv[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) tv[u] = *reinterpret_cast<const float4 *>(tcol + (i + u) * 16);
+                        const float dvv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            acc.x = fmaf(dvv[u], tv[u].x, acc.x); acc.y = fmaf(dvv[u], tv[u].y, acc.y);
+                            acc.z = fmaf(dvv[u], tv[u].z, acc.z); acc.w = fmaf(dvv[u], tv[u].w, acc.w);
+                        }
+                    }
+                    *reinterpret_cast<float4 *>(Mf + (16 * r + tt) * kLd + 16 * c + 4 * lg) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
+                }
+                named_bar_sync(1, 128);
+            }
+            // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
+            unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
+            if (x < kC) {
+                const int t = x;
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    float v[16];
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4) {
+                        const int i = 16 * q + c;
+                        const float4 mv = (i >> 4) <= (t >> 4) ? *reinterpret_cast<const float4 *>(Mf + t * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        v[c] = mv.x; v[c + 1] = mv.y; v[c + 2] = mv.z; v[c + 3] = mv.w;
+                    }
+                    store_row_chunks(mpm, t, 2 * q, v);
+                }
+            }
+            fence_async_smem();
+            mbar_arrive(&bars.m_ready);
+            mbar_arrive(&bars.inv_done[b & 1]);
+            // ---- PM rows (lanes 0..63 of the (6) accumulator) -> rows 64..127 of [M; PM]
+            mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            if (x < kC) {
+#pragma unroll 1
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t rr[16];
+                    tmem_ld16(lane_base + kTmPM + 16 * q, rr);
+                    tmem_ld_wait();
+                    float v[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
+                    store_row_chunks(mpm, kC + x, 2 * q, v);
+                }
+            }
+            fence_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars.mpm_ready[b & 1]);
+        }
+    } else if (warp >= 8) {
+        // ======================================================= out warpgroup: o_t[j] = scale (gam_t (S^T q_t)_j + (P u)_t[j]); lane = j
+        const int j = tid - 256;
+        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
+        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
+        const int x = j;   // TMEM lane: 0..63 rows of Q K^T (-> P), 64..127 rows of K K^T (-> A)
+        // epilogue of (1) for block b: P (bf16 operand of (6)) and A (fp32, input of the inverse)
+        auto g_epilogue = [&](int b) {
+            const float *sc = gb + (b & 1) * kGbFloats;
+            mbar_wait(&bars.gb_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
+            if (x < kC) {
+                // the P buffer is free once (6) of block b-1 has read it
+                if (b >= 1) mbar_wait(&bars.pm_done, (b - 1) & 1, &dead, a.status);
+            } else {
+                // the A buffer of this parity is free once block b-2 has been inverted
+                if (b >= 2) mbar_wait(&bars.inv_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+            }
             mbar_wait(&bars.g_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
             {
@@ -319,101 +469,17 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
             }
             tc_fence_before_sync();
-            named_bar_sync(1, 128);
-            // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k.
             if (x < kC) {
-                const int k = x >> 4, c = x & 15;
-                const float *Ab = Af + (16 * k) * kLd + 16 * k;
-                float xv[16];
-#pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    float acc = (t == c) ? 1.f : 0.f;
-#pragma unroll
-                    for (int i = 0; i < t; ++i) acc = fmaf(-Ab[t * kLd + i], xv[i], acc);
-                    xv[t] = (t >= c) ? acc : 0.f;
-                }
-#pragma unroll
-                for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
+                fence_async_smem();
+                mbar_arrive(&bars.p_ready);
+            } else {
+                mbar_arrive(&bars.a_ready);
             }
-            named_bar_sync(1, 128);
-            // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc.
-            // A thread owns a 1 x 4 strip (row tt, columns 4*lg..4*lg+3) of a 16 x 16 block.
-            for (int d = 1; d < 4; ++d) {
-                const int nstrip = (4 - d) * 64;
-                for (int e = x; e < nstrip; e += 128) {
-                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *arow = Af + (16 * r + tt) * kLd;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int ii = 16 * c; ii < 16 * r; ++ii) {
-                        const float av = arow[ii];
-                        const float4 mv = *reinterpret_cast<const float4 *>(Mf + ii * kLd + 16 * c + 4 * lg);
-                        acc.x = fmaf(av, mv.x, acc.x); acc.y = fmaf(av, mv.y, acc.y);
-                        acc.z = fmaf(av, mv.z, acc.z); acc.w = fmaf(av, mv.w, acc.w);
-                    }
-                    *reinterpret_cast<float4 *>(Tt + c * 256 + tt * 16 + 4 * lg) = acc;
-                }
-                named_bar_sync(1, 128);
-                for (int e = x; e < nstrip; e += 128) {
-                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *drow = Mf + (16 * r + tt) * kLd + 16 * r;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-                    for (int i = 0; i < 16; ++i) {
-                        const float dv = drow[i];
-                        const float4 tv = *reinterpret_cast<const float4 *>(Tt + c * 256 + i * 16 + 4 * lg);
-                        acc.x = fmaf(dv, tv.x, acc.x); acc.y = fmaf(dv, tv.y, acc.y);
-                        acc.z = fmaf(dv, tv.z, acc.z); acc.w = fmaf(dv, tv.w, acc.w);
-                    }
-                    *reinterpret_cast<float4 *>(Mf + (16 * r + tt) * kLd + 16 * c + 4 * lg) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
-                }
-                named_bar_sync(1, 128);
-            }
-            // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
-            unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
-            if (x < kC) {
-                const int t = x;
-#pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    float v[16];
-#pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        const int i = 16 * q + c;
-                        const float4 mv = (i >> 4) <= (t >> 4) ? *reinterpret_cast<const float4 *>(Mf + t * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        v[c] = mv.x; v[c + 1] = mv.y; v[c + 2] = mv.z; v[c + 3] = mv.w;
-                    }
-                    store_row_chunks(mpm, t, 2 * q, v);
-                }
-            }
-            fence_async_smem();
-            mbar_arrive(&bars.m_ready);
-            // ---- PM rows (lanes 0..63 of the (6) accumulator) -> rows 64..127 of [M; PM]
-            mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            if (x < kC) {
-#pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t rr[16];
-                    tmem_ld16(lane_base + kTmG + 16 * q, rr);
-                    tmem_ld_wait();
-                    float v[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
-                    store_row_chunks(mpm, kC + x, 2 * q, v);
-                }
-            }
-            fence_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&bars.mpm_ready[b & 1]);
-        }
-    } else if (warp >= 8) {
-        // ======================================================= out warpgroup: o_t[j] = scale (gam_t (S^T q_t)_j + (P u)_t[j]); lane = j
-        const int j = tid - 256;
-        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
-        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
+        };
+        g_epilogue(0);
         for (int b = 0; b < nblk; ++b) {
+            if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
             const float *sc = gb + (b & 1) * kGbFloats;
-            mbar_wait(&bars.gb_ready[b & 1], (b >> 1) & 1, &dead, a.status);
             mbar_wait(&bars.d1_done, b & 1, &dead, a.status);
             mbar_wait(&bars.up_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
