@@ -6,6 +6,7 @@ workload, single-state initialisation, exact composition, and the chunkwise scan
 recompute segment from the composed state (both families when the workload has both).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg3|cfg4] [--impl reference]
+    python bench.py --sweep        # microseconds per exact composition against K (a JSON line of its own)
 
 Prints ONE JSON line (rank 0).  `value` = context tokens served per second by the step (all requests'
 context tokens / step time), device-timed with inputs resident in HBM; `e2e` = the same with every
@@ -56,6 +57,11 @@ def gdn_scan_flops(tokens: int, s=GDN_SHAPE, C=GDN_BLOCK) -> float:
 def ssd_scan_flops(tokens: int, s=SSD_SHAPE, Q=SSD_BLOCK) -> float:
     """Chunkwise SSD flops: per token and head 2*(2 N P + Q P) plus C B^T once per group 2*Q*N."""
     return (2.0 * (2 * s["N"] * s["P"] + Q * s["P"]) * s["H"] + 2.0 * Q * s["N"] * s["G"]) * tokens
+
+
+# DRAM bytes (read + write) per scanned token from the ncu capture of one 16384-token launch of each scan kernel
+# (8 sequences x 2048 tokens); the traffic of a scan grows in proportion to its tokens.
+NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.03e6 + 119.80e6) / 16384, "mamba2.scan": None}
 
 
 def gdn_scan_bytes(tokens: int, s=GDN_SHAPE) -> float:
@@ -193,10 +199,10 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def cpu_baseline_sample(seconds_hint: float = 15.0):
+def cpu_baseline_sample(pairs: int = 8):
     """The oracle as it stands, timed on this machine's cores on a bounded sample of the workload:
-    exact composition of one GDN request (K = 16) plus a 12288-token GDN scan, all 32 value heads,
-    and the same for one Mamba-2 request (K = 16, 12288 tokens, 80 heads)."""
+    `pairs` times, exact composition of one GDN request (K = 16) plus a 12288-token GDN scan, all 32 value
+    heads, and the same for one Mamba-2 request (K = 16, 12288 tokens, 80 heads)."""
     import oracle
     rng = np.random.default_rng(99)
     s, m = GDN_SHAPE, SSD_SHAPE
@@ -210,16 +216,17 @@ def cpu_baseline_sample(seconds_hint: float = 15.0):
     lam = wl.synthetic_logdecay(rng, K, m["H"])
     oracle.num_threads()
     t0 = time.perf_counter()
-    S0 = oracle.init_exact_gdn(states, trans)
-    oracle.gdn_seq(tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], S0)
-    M0 = oracle.init_exact_mamba(mstates, lam)
-    oracle.ssd_seq(mt["x"], mt["dt"], A, mt["B"], mt["C"], M0)
+    for _ in range(pairs):
+        S0 = oracle.init_exact_gdn(states, trans)
+        oracle.gdn_seq(tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], S0)
+        M0 = oracle.init_exact_mamba(mstates, lam)
+        oracle.ssd_seq(mt["x"], mt["dt"], A, mt["B"], mt["C"], M0)
     dt = time.perf_counter() - t0
     # context covered by the sample at the workload's recompute ratio (0.2): each request's
     # T recomputed tokens stand for T / 0.2 context tokens
-    context = 2 * T / 0.2
+    context = pairs * 2 * T / 0.2
     return dict(value=context / dt, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
-                sample=f"1 GDN + 1 Mamba-2 request, K={K} exact composition + {T}-token scan each "
+                sample=f"{pairs} GDN + {pairs} Mamba-2 requests, K={K} exact composition + {T}-token scan each "
                        f"(= {int(context)} context tokens at r=0.2), {dt:.2f} s"), dt
 
 
@@ -228,13 +235,14 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    pairs = 2
     for _ in range(args.warmup if args.warmup < 2 else 1):
-        cpu_baseline_sample()
+        cpu_baseline_sample(pairs)
     times, base = [], None
     for _ in range(args.steps):
-        base, dt = cpu_baseline_sample()
+        base, dt = cpu_baseline_sample(pairs)
         times.append(dt)
-    context = 2 * 12288 / 0.2
+    context = pairs * 2 * 12288 / 0.2
     t = sum(times) / len(times)
     value = context / t
     base["value"] = value
@@ -340,14 +348,15 @@ def run_ours(args):
             f.step()
             f.download()
 
+    # clocks are sampled from the warm-up to the end of the end-to-end steps: the GPU is busy throughout
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     g_step = graph_of(step)
     for _ in range(max(args.warmup, 3)):
         g_step.replay()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     if cold_by_size:
         ms = timed_back_to_back(g_step.replay, args.steps)
     else:
@@ -358,10 +367,10 @@ def run_ours(args):
         for name, fn in (("init_last", f.init_last), ("init_exact", f.init_exact), ("scan", f.scan)):
             g = graph_of(fn)
             parts[f"{f.fam}.{name}"] = timed_flushed(g.replay, max(args.steps, 5), reduce="median")
-    clocks = sampler.stop() if rank == 0 else None
     e2e_steps = max(1, min(args.steps, 3))
     step_e2e()
     ms_e2e = timed_back_to_back(step_e2e, e2e_steps)
+    clocks = sampler.stop() if rank == 0 else None
 
     if world > 1:
         job_context_tokens = sharding.job_total(context_tokens, dist, "cuda")
@@ -388,8 +397,11 @@ def run_ours(args):
         flops = gdn_scan_flops(f.scan_tokens) if fam_name == "gdn" else ssd_scan_flops(f.scan_tokens)
         achieved = flops / (parts[dom] * 1e-3) / 1e12
         peak = peaks["bf16_tflops_sustained"] if parts[dom] > 50.0 else peaks["bf16_tflops"]
-        roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
-                    kernel=dom, peak_source=peak_src)
+        per_token = NCU_DRAM_BYTES_PER_TOKEN.get(dom)
+        roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
+                    traffic=None if per_token is None else per_token * f.scan_tokens,
+                    traffic_source="ncu dram bytes of a 16384-token launch, scaled by tokens", kernel=dom,
+                    peak_source=peak_src)
     else:
         nbytes = f.pool_bytes_unique + f.S0.numel() * 4
         achieved = nbytes / (parts[dom] * 1e-3) / 1e9
@@ -431,6 +443,69 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """--sweep: microseconds per exact composition against K, both families, batch 1 and batch 8 (every request
+    with its own pool entries), L2 flushed before every timed launch.  Prints one JSON line of its own."""
+    import torch
+
+    from paper_2608_11231_b200 import binding as b
+    torch.cuda.set_device(0)
+    b.load()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            hbm = json.load(fh)["hbm_gbs"]
+    except OSError:
+        hbm = 6650.0
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    rows = []
+    for fam in ("mamba2", "gdn"):
+        if fam == "gdn":
+            H, dk, dv, code = GDN_SHAPE["H_v"], GDN_SHAPE["d_k"], GDN_SHAPE["d_v"], b.LKV_FAMILY_GDN
+        else:
+            H, dk, dv, code = SSD_SHAPE["H"], SSD_SHAPE["N"], SSD_SHAPE["P"], b.LKV_FAMILY_MAMBA2
+        for n_req in (1, 8):
+            for K in (1, 2, 4, 8, 16, 32, 64):
+                n_pool = n_req * K
+                states = torch.randn((n_pool, H, dk, dv), generator=gen, device="cuda")
+                if fam == "gdn":
+                    trans = torch.randn((n_pool, H, dk, dk), generator=gen, device="cuda") * (0.45 / dk ** 0.5)
+                else:
+                    trans = -2.0 * torch.rand((n_pool, H), generator=gen, device="cuda")
+                ids = np.arange(n_pool, dtype=np.int32)
+                cu_k = (np.arange(n_req + 1) * K).astype(np.int32)
+                S0 = torch.empty((n_req, H, dk, dv), device="cuda")
+                ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+
+                def fn():
+                    b.lkv_init_state_batched(states, trans, ids, cu_k, n_req, b.LKV_INIT_EXACT, None, S0,
+                                             family=code, workspace_t=ws)
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    fn()
+                ts = []
+                for _ in range(max(args.steps, 7)):
+                    flush_buf.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    g.replay()
+                    e1.record()
+                    e1.synchronize()
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+                us = statistics.median(ts)
+                nbytes = (states.numel() + S0.numel()) * 4 + trans.numel() * 4
+                if fam == "gdn":   # the first chunk's transition is never read
+                    nbytes -= n_req * H * dk * dk * 4
+                rows.append(dict(family=fam, requests=n_req, K=K, us=round(us, 2), gbs=round(nbytes / us / 1e3, 1),
+                                 frac_of_hbm=round(nbytes / us / 1e3 / hbm, 3)))
+                del states, trans, S0
+    print(json.dumps(dict(sweep="compose_us_vs_K", timing="graph replay of one launch between CUDA events (includes "
+                          "about 2 us of launch gap), L2 flushed before each, median", rows=rows)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -438,8 +513,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="composition time against K instead of the step benchmark")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -6,7 +6,7 @@
 // TMEM lanes): lane j owns state column j.  Per block, with cg the running sum of g,
 // gam_t = e^{cg_t}, Gam_ti = e^{cg_t - cg_i}, w_i = e^{cg_C - cg_i} and S the incoming state:
 //   (1) G    = [Q;K] K^T             rows 0..63: q_t.k_i, rows 64..127: k_t.k_i           tcgen05
-//       P_ti = Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)             prep warps
+//       P_ti = Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)             out warps
 //       M    = (I + A)^{-1}          (UT transform: 16x16 diagonal blocks by substitution,
 //                                     off-diagonal blocks by block products, fp32)        prep warps
 //   (6) PM   = P M                                                                        tcgen05
@@ -16,8 +16,9 @@
 //       o_t  = scale (gam_t S^T q_t + (P u)_t)                                            out warps
 //   (5) S^T <- gam_C S^T + (U o w)^T K   fp32 state accumulated in TMEM (pre-scaled there) tcgen05
 //       and a bf16 copy of S^T in shared memory is the A operand of (2) for the next block.
-// The prep warps work one block ahead of the chain, so (1), the inverse and (6) are off the
-// block-to-block chain (2) -> r -> (3) -> U o w -> (5) -> state copy.
+// The prep warps (cumulative decay, the inverse, the bf16 [M; PM] operand) and the mask epilogue of (1)
+// work one block ahead of the chain, so (1), the inverse and (6) are off the block-to-block chain
+// (2) -> r -> (3) -> U o w -> (5) -> state copy.
 // A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
 // Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 out,
 // 12-15 prep, 16 TMA, 17 MMA issue.  All waits on mbarriers are bounded.

@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _error_log(request):
+    """With LKV_ERR_LOG=<file>, append every test's measured max-relative errors to that file."""
+    import helpers
+    helpers.ERRORS.clear()
+    yield
+    path = os.environ.get("LKV_ERR_LOG")
+    if path and helpers.ERRORS:
+        with open(path, "a") as fh:
+            fh.write(request.node.nodeid + " " + " ".join(f"{e:.3e}" for e in helpers.ERRORS) + "\n")

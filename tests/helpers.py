@@ -11,14 +11,18 @@ TOL_F32 = 1e-4
 TOL_BF16 = 2e-2
 
 
+# every maxrel() value of the running test, in call order (conftest.py writes them out on request)
+ERRORS: list = []
+
+
 def maxrel(x, ref) -> float:
     """max |x - ref| / max |ref| over one tensor (elementwise-relative is undefined at zeros)."""
     x = np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     den = np.abs(ref).max()
-    if den == 0.0:
-        return float(np.abs(x).max())
-    return float(np.abs(x - ref).max() / den)
+    err = float(np.abs(x).max()) if den == 0.0 else float(np.abs(x - ref).max() / den)
+    ERRORS.append(err)
+    return err
 
 
 def frobrel(x, ref) -> float:
