@@ -4,16 +4,19 @@
 // a bf16 copy in shared memory as an MMA operand).  With l the running sum of dt * A_h inside the
 // block and S the incoming state, per block:
 //   (a) G      = C B^T                                   [128 x 128], K = N                 tcgen05
-//       G'_ti  = G_ti e^{l_t - l_i} dt_i  (i <= t), 0 otherwise -> bf16 operand             epilogue warps
-//   (b) Yintra = G' X                                    [128 x 64],  K = 128 tokens         tcgen05
+//       G'_ti  = G_ti e^{l_t - l_i} dt_i  (i <= t), 0 otherwise -> bf16 operand in TMEM     epilogue warps
+//   (b) Yintra = G' X                                    [128 x 64],  K = 128 tokens         tcgen05 (A from TMEM)
 //   (c) Yinter = C S                                     [128 x 64],  K = N                  tcgen05
 //       y_t    = Yintra_t + e^{l_t} Yinter_t                                                 epilogue warps
 //   (d) S     <- e^{l_Q} S + B^T X~,  X~_i = e^{l_Q - l_i} dt_i x_i   [128 x 64], K = tokens   tcgen05
 //       (the state is pre-scaled in tensor memory, (d) accumulates onto it)                  state warps
-// Only (c) depends on the previous block, so the tensor pipe and the SIMT warps overlap freely;
-// the block-to-block chain is (d) -> state copy -> (c).  A padded token has dt = 0.
-// Warps 0-7 epilogue (thread = token row, warpgroup = column half), 8-11 state and per-block
-// scalars, 12 TMA, 13 MMA issue.  All waits on mbarriers are bounded.
+// Only (c) and (d) depend on the previous block: (a) of the next block is issued as soon as the mask
+// epilogue has drained G, so the epilogue warps never wait for the block-to-block chain
+// (d) -> state copy -> (c), (d); the scaled X~ of the next block is prepared while (d) runs.
+// A padded token has dt = 0.
+// Warps 0-7 epilogue (thread = token row, warpgroup = column half), 8-11 state copy (the only SIMT
+// work on the block-to-block chain), 12-15 per-block scalars and X~ (running ahead of the chain),
+// 16 TMA, 17 MMA issue.  All waits on mbarriers are bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -26,33 +29,36 @@ using namespace tc;
 constexpr int kP = 64;     // headdim
 constexpr int kN = 128;    // d_state
 constexpr int kQ = 128;    // tokens per block
-constexpr int kThreads = 448;
+constexpr int kThreads = 576;
 
 // shared-memory map (bytes, after 1024-byte alignment); every tile row is 128 bytes, 128-byte swizzle
 constexpr int kXTile = kQ * 128;            // X [128 tokens x 64 p]
 constexpr int kBTile = 2 * kQ * 128;        // B [B_kb0 | B_kb1], each [128 tokens x 64 n]
-constexpr int kCTile = 2 * kQ * 128;        // C likewise; reused for G' once (a) and (c) are done
+constexpr int kCTile = 2 * kQ * 128;        // C likewise
 constexpr int kStageBytes = kXTile + kBTile + kCTile;   // 80 KB
-constexpr int kOffX2 = 2 * kStageBytes;     // X~ [128 tokens x 64 p]
-constexpr int kOffHb = kOffX2 + kXTile;     // bf16 state [128 n x 64 p]
-constexpr int kOffSc = kOffHb + kN * 128;   // per-block scalars, double-buffered
+constexpr int kOffX2 = 2 * kStageBytes;     // X~ [128 tokens x 64 p], double-buffered
+constexpr int kOffHb = kOffX2 + 2 * kXTile; // bf16 state [128 n x 64 p]
+constexpr int kOffSc = kOffHb + kN * 128;   // per-block scalars, three buffers
 constexpr int kScFloats = 5 * kQ + 4;       // l2 = l log2(e), e^{l}, s = e^{l_Q - l} dt, f = e^{l_ref - l} dt, dt, flag
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxGroupRange = 100.f;     // log2 units: above this the per-group factors could overflow
-constexpr int kSmemBytes = kOffSc + 2 * kScFloats * 4 + 1024;
+constexpr int kSmemBytes = kOffSc + 3 * kScFloats * 4 + 1024;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 // tensor-memory map (columns)
 constexpr uint32_t kTmG = 0;        // 128
 constexpr uint32_t kTmYa = 128;     // Yintra, 2 x 64
 constexpr uint32_t kTmYe = 256;     // Yinter, 2 x 64
 constexpr uint32_t kTmH = 384;      // 64
+constexpr uint32_t kTmGp = 448;     // G' as bf16 pairs: 128 K-elements in 64 columns
 constexpr uint32_t kTmemCols = 512;
 
 struct Bars {
-    uint64_t full[2], tiles_free[2];
-    uint64_t ac_done, y_done, h_done;                  // tcgen05.commit targets
-    uint64_t mg_ready, yo_done[2];                     // 256 epilogue threads
-    uint64_t sc_ready[2], x2_ready, hb_ready;          // 128 state threads
+    uint64_t full_bc[2], full_x[2];                    // TMA transactions
+    uint64_t bc_free[2], ac_done, y_done, h_done[2];   // tcgen05.commit targets
+    uint64_t x_free[2];                                // the epilogue thread that stores y out of the X tile
+    uint64_t mg_ready, yo_done[3];                     // 256 epilogue threads
+    uint64_t sc_ready[3], x2_ready[2], hb_ready;       // 128 threads (scalar warps; hb_ready: state warps)
 };
 
 __device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
@@ -68,7 +74,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant__ CUtensorMap mapX,
-                       const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC) {
+                       const __grid_constant__ CUtensorMap mapB, const __grid_constant__ CUtensorMap mapC,
+                       const __grid_constant__ CUtensorMap mapY) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ Bars bars;
@@ -90,96 +97,118 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
     }
     if (tid == 0) {
         dead = 0;
-        uint64_t *b1 = &bars.full[0];
-        for (int i = 0; i < 7; ++i) mbar_init(b1 + i, 1);
+        uint64_t *b1 = &bars.full_bc[0];
+        for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
         uint64_t *b256 = &bars.mg_ready;
-        for (int i = 0; i < 3; ++i) mbar_init(b256 + i, 256);
+        for (int i = 0; i < 4; ++i) mbar_init(b256 + i, 256);
         uint64_t *b128 = &bars.sc_ready[0];
-        for (int i = 0; i < 4; ++i) mbar_init(b128 + i, 128);
+        for (int i = 0; i < 6; ++i) mbar_init(b128 + i, 128);
         mbar_fence_init();
     }
-    if (warp == 13) tmem_alloc(&tmem_base, kTmemCols);
+    if (warp == 17) tmem_alloc(&tmem_base, kTmemCols);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_base;
     float *scal = reinterpret_cast<float *>(sm + kOffSc);
 
-    if (warp == 12) {
+    if (warp == 16) {
         // ======================================================= TMA producer
         if (lane == 0) {
             tma_prefetch_desc(&mapX);
             tma_prefetch_desc(&mapB);
             tma_prefetch_desc(&mapC);
+            tma_prefetch_desc(&mapY);
             for (int b = 0; b < nblk; ++b) {
+                // B and C of block b-2 are free after its (d); its X tile, which also stages y, after y has left it
                 const int st = b & 1;
-                if (b >= 2) mbar_wait(&bars.tiles_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
                 unsigned char *base = sm + st * kStageBytes;
                 const int row = t_begin + b * kQ;
-                mbar_expect_tx(&bars.full[st], kStageBytes);
-                tma_load_2d(base, &mapX, h * kP, row, &bars.full[st]);
+                if (b >= 2) mbar_wait(&bars.bc_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                mbar_expect_tx(&bars.full_bc[st], kBTile + kCTile);
                 for (int kb = 0; kb < 2; ++kb) {
-                    tma_load_2d(base + kXTile + kb * kQ * 128, &mapB, grp * kN + kb * 64, row, &bars.full[st]);
-                    tma_load_2d(base + kXTile + kBTile + kb * kQ * 128, &mapC, grp * kN + kb * 64, row, &bars.full[st]);
+                    tma_load_2d(base + kXTile + kb * kQ * 128, &mapB, grp * kN + kb * 64, row, &bars.full_bc[st]);
+                    tma_load_2d(base + kXTile + kBTile + kb * kQ * 128, &mapC, grp * kN + kb * 64, row, &bars.full_bc[st]);
                 }
+                if (b >= 2) mbar_wait(&bars.x_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                mbar_expect_tx(&bars.full_x[st], kXTile);
+                tma_load_2d(base, &mapX, h * kP, row, &bars.full_x[st]);
             }
         }
-    } else if (warp == 13) {
+    } else if (warp == 17) {
         // ======================================================= MMA issuer (one elected thread)
         if (elect_one()) {
             constexpr uint32_t idA = umma_idesc(kFmtBF16, false, false, 128, 128);   // (a): C, B both K-major
             constexpr uint32_t idC = umma_idesc(kFmtBF16, false, true, 128, 64);     // (c), (b): B operand MN-major
             constexpr uint32_t idD = umma_idesc(kFmtBF16, true, true, 128, 64);      // (d): both MN-major
             const uint64_t dHb = umma_desc(smem_u32(sm + kOffHb), 0, 1024);
-            const uint64_t dX2 = umma_desc(smem_u32(sm + kOffX2), 0, 1024);
-            for (int b = 0; b < nblk; ++b) {
-                const uint32_t par = b & 1;
+            // (a) G = C B^T of block b (both operands K-major)
+            auto issue_a = [&](int b) {
                 const uint32_t sbase_u = smem_u32(sm + (b & 1) * kStageBytes);
-                const uint64_t dX = umma_desc(sbase_u, 0, 1024);
-                const uint64_t dBk = umma_desc(sbase_u + kXTile, 0, 1024);                 // B tile, K-major view
-                const uint64_t dBm = umma_desc(sbase_u + kXTile, kQ * 128, 1024);          // B tile, MN-major view (n blocks 16 KB apart)
-                const uint64_t dCk = umma_desc(sbase_u + kXTile + kBTile, 0, 1024);        // C tile, later G'
-                mbar_wait(&bars.full[b & 1], (b >> 1) & 1, &dead, a.status);
-                mbar_wait(&bars.hb_ready, par, &dead, a.status);
-                if (b >= 2) mbar_wait(&bars.yo_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                tc_fence_after_sync();
-                // (c) Yinter = C S : A = C (K = n), B = bf16 state read MN-major (rows = n)
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tm + kTmYe + 64 * par, dCk + (((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4), dHb + ((k * 16 * 128) >> 4), idC, k > 0);
-                // (a) G = C B^T
+                const uint64_t dBk = umma_desc(sbase_u + kXTile, 0, 1024);
+                const uint64_t dCk = umma_desc(sbase_u + kXTile + kBTile, 0, 1024);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     const uint64_t off = ((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4;
                     umma_bf16(tm + kTmG, dCk + off, dBk + off, idA, k > 0);
                 }
                 umma_commit(&bars.ac_done);
+            };
+            mbar_wait(&bars.full_bc[0], 0, &dead, a.status);
+            tc_fence_after_sync();
+            issue_a(0);
+            for (int b = 0; b < nblk; ++b) {
+                const uint32_t par = b & 1;
+                const uint32_t sbase_u = smem_u32(sm + (b & 1) * kStageBytes);
+                const uint64_t dX = umma_desc(sbase_u, 0, 1024);
+                const uint64_t dBm = umma_desc(sbase_u + kXTile, kQ * 128, 1024);          // B tile, MN-major view (n blocks 16 KB apart)
+                const uint64_t dCk = umma_desc(sbase_u + kXTile + kBTile, 0, 1024);
+                const uint64_t dX2 = umma_desc(smem_u32(sm + kOffX2 + (b & 1) * kXTile), 0, 1024);
+                mbar_wait(&bars.hb_ready, par, &dead, a.status);
+                if (b >= 2) mbar_wait(&bars.yo_done[(b - 2) % 3], ((b - 2) / 3) & 1, &dead, a.status);
+                tc_fence_after_sync();
+                // (c) Yinter = C S : A = C (K = n), B = bf16 state read MN-major (rows = n)
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tm + kTmYe + 64 * par, dCk + (((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4), dHb + ((k * 16 * 128) >> 4), idC, k > 0);
                 // (d) S += B^T X~ : A = B tile read MN-major (rows = tokens), B = X~ read MN-major
-                mbar_wait(&bars.x2_ready, par, &dead, a.status);
+                mbar_wait(&bars.x2_ready[b & 1], (b >> 1) & 1, &dead, a.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     umma_bf16(tm + kTmH, dBm + ((k * 16 * 128) >> 4), dX2 + ((k * 16 * 128) >> 4), idD, true);
-                umma_commit(&bars.h_done);
-                // (b) Yintra = G' X : A = G' (in the C buffer, K = tokens), B = X read MN-major
+                umma_commit(&bars.h_done[b & 1]);
+                umma_commit(&bars.bc_free[b & 1]);
+                // (b) Yintra = G' X : A = G' from tensor memory (8 columns per K-step of 16 tokens), B = X read MN-major
                 mbar_wait(&bars.mg_ready, par, &dead, a.status);
+                mbar_wait(&bars.full_x[b & 1], (b >> 1) & 1, &dead, a.status);
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    umma_bf16(tm + kTmYa + 64 * par, dCk + (((k >> 2) * (kQ * 128) + (k & 3) * 32) >> 4), dX + ((k * 16 * 128) >> 4), idC, k > 0);
+                    umma_bf16_ts(tm + kTmYa + 64 * par, tm + kTmGp + 8 * k, dX + ((k * 16 * 128) >> 4), idC, k > 0);
                 umma_commit(&bars.y_done);
-                umma_commit(&bars.tiles_free[b & 1]);
+                // (a) of the next block: G has been drained by the mask epilogue of this one
+                if (b + 1 < nblk) {
+                    mbar_wait(&bars.full_bc[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+                    issue_a(b + 1);
+                }
             }
         }
-    } else if (warp >= 8) {
-        // ======================================================= state warpgroup: thread = token (scalars, X~) / state row n
-        const int x = tid - 256;   // 0..127
-        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    } else if (warp >= 12) {
+        // ======================================================= scalar warpgroup: thread = token; per-block scalars and X~, ahead of the chain
+        const int x = tid - 384;   // 0..127
         const float Ah = a.A[h];
-        auto prepare_scalars = [&](int b) {
-            float *dst = scal + (b & 1) * kScFloats;
+        // dt of this thread's token in block b (0 beyond the sequence end); fetched one block before it is used
+        auto fetch_dt = [&](int b) {
             const int t = t_begin + b * kQ + x;
-            const float dtv = (t < t_end) ? a.dt[static_cast<size_t>(t) * a.H + h] : 0.f;
+            return (b < nblk && t < t_end) ? a.dt[static_cast<size_t>(t) * a.H + h] : 0.f;
+        };
+        float dt_next = fetch_dt(0);
+        auto prepare_scalars = [&](int b) {
+            float *dst = scal + (b % 3) * kScFloats;
+            const float dtv = dt_next;
+            dt_next = fetch_dt(b + 1);
             float run = dtv * Ah;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -204,10 +233,43 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             named_bar_sync(1, 128);
             if (x == 0) dst[5 * kQ] = scan_carry[0] + scan_carry[1] + scan_carry[2] + scan_carry[3];
             named_bar_sync(1, 128);
-            mbar_arrive(&bars.sc_ready[b & 1]);
+            mbar_arrive(&bars.sc_ready[b % 3]);
         };
-        prepare_scalars(0);
+        // X~ row of token x of block b: s_x * X[x][:]
+        auto scaled_x = [&](int b) {
+            const float *sc = scal + (b % 3) * kScFloats;
+            mbar_wait(&bars.full_x[b & 1], (b >> 1) & 1, &dead, a.status);
+            const unsigned char *xt = sm + (b & 1) * kStageBytes;
+            unsigned char *x2 = sm + kOffX2 + (b & 1) * kXTile;
+            const float s = sc[2 * kQ + x];
+#pragma unroll
+            for (int c8 = 0; c8 < 8; ++c8) {
+                const uint32_t off = sw128_offset(x, c8);
+                const uint4 v = *reinterpret_cast<const uint4 *>(xt + off);
+                const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    w[e] = pack_bf16(__uint_as_float(in[e] << 16) * s, __uint_as_float(in[e] & 0xFFFF0000u) * s);
+                *reinterpret_cast<uint4 *>(x2 + off) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            fence_async_smem();
+            mbar_arrive(&bars.x2_ready[b & 1]);
+        };
+        for (int b = 0; b < nblk; ++b) {
+            // the scalar buffer of block b is the one block b-3 used: its outputs must be written
+            if (b >= 3) mbar_wait(&bars.yo_done[b % 3], ((b - 3) / 3) & 1, &dead, a.status);
+            prepare_scalars(b);
+            // the X~ buffer of block b was read by (d) of block b-2
+            if (b >= 2) mbar_wait(&bars.h_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+            scaled_x(b);
+        }
+    } else if (warp >= 8) {
+        // ======================================================= state warpgroup: thread = state row n
+        const int x = tid - 256;   // 0..127
+        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         // initial state: fp32 into tensor memory pre-scaled by e^{l_Q} of block 0, bf16 copy unscaled
+        mbar_wait(&bars.sc_ready[0], 0, &dead, a.status);
         {
             const float gq = scal[kQ + kQ - 1];
 #pragma unroll
@@ -234,36 +296,12 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             mbar_arrive(&bars.hb_ready);
         }
         for (int b = 0; b < nblk; ++b) {
-            const float *sc = scal + (b & 1) * kScFloats;
-            // X~ row of token x: s_x * X[x][:]
-            mbar_wait(&bars.full[b & 1], (b >> 1) & 1, &dead, a.status);
-            {
-                const unsigned char *xt = sm + (b & 1) * kStageBytes;
-                const float s = sc[2 * kQ + x];
-#pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) {
-                    const uint32_t off = sw128_offset(x, c8);
-                    const uint4 v = *reinterpret_cast<const uint4 *>(xt + off);
-                    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
-                    uint32_t w[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        w[e] = pack_bf16(__uint_as_float(in[e] << 16) * s, __uint_as_float(in[e] & 0xFFFF0000u) * s);
-                    *reinterpret_cast<uint4 *>(sm + kOffX2 + off) = make_uint4(w[0], w[1], w[2], w[3]);
-                }
-            }
-            fence_async_smem();
-            mbar_arrive(&bars.x2_ready);
-            if (b + 1 < nblk) {
-                // the scalar buffer of block b+1 is the one block b-1 used: its outputs must be written
-                if (b >= 1) mbar_wait(&bars.yo_done[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
-                prepare_scalars(b + 1);
-            }
             // state after (d): copy for the next block's (c), pre-scale for its (d); or S_T at the end
-            mbar_wait(&bars.h_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
             const bool last = b + 1 == nblk;
-            const float gq = last ? 1.f : scal[((b + 1) & 1) * kScFloats + kQ + kQ - 1];
+            if (!last) mbar_wait(&bars.sc_ready[(b + 1) % 3], ((b + 1) / 3) & 1, &dead, a.status);
+            const float gq = last ? 1.f : scal[((b + 1) % 3) * kScFloats + kQ + kQ - 1];
+            mbar_wait(&bars.h_done[b & 1], (b >> 1) & 1, &dead, a.status);
+            tc_fence_after_sync();
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 uint32_t rr[32];
@@ -303,16 +341,16 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(a.y);
         for (int b = 0; b < nblk; ++b) {
-            const float *sc = scal + (b & 1) * kScFloats;
-            mbar_wait(&bars.sc_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            const float *sc = scal + (b % 3) * kScFloats;
+            mbar_wait(&bars.sc_ready[b % 3], (b / 3) & 1, &dead, a.status);
             mbar_wait(&bars.ac_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
-            // G' row t, columns i = 64*half .. 64*half+63 -> K-block `half` of the operand in the C buffer.
+            // G' row t, columns i = 64*half .. 64*half+63 -> bf16 pairs in TMEM columns 32*half .. 32*half+31 of the operand.
+            // ((b) of the previous block, which read that operand, completed before its y epilogue ran.)
             // e^{l_t - l_i} dt_i = 2^{l2_t - l2_ref} * f_i with ref the first column of i's group of 16: one
             // exponential per group instead of one per element (every factor is <= 1 where i <= t);
             // blocks whose decay is too violent for that take the per-element path.
             {
-                unsigned char *gk = sm + (b & 1) * kStageBytes + kXTile + kBTile + half * (kQ * 128);
                 const float lt = sc[t];
                 const bool fast = sc[5 * kQ] == 0.f;
 #pragma unroll 1
@@ -343,11 +381,10 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                             w[c / 2] = pack_bf16(v0, v1);
                         }
                     }
-                    *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 2 * q)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(gk + sw128_offset(t, 2 * q + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+                    tmem_st8(lane_base + kTmGp + 32 * half + 8 * q, w);
                 }
             }
-            fence_async_smem();
+            tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(&bars.mg_ready);
             // y_t[p] = Yintra + e^{l_t} Yinter, p = 32*half .. 32*half+31
@@ -359,29 +396,47 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 tmem_ld32(lane_base + kTmYe + 64 * (b & 1) + 32 * half, ye);
                 tmem_ld_wait();
                 const float et = sc[kQ + t];
-                const int tok = t_begin + b * kQ + t;
-                if (tok < t_end) {
-                    __nv_bfloat16 *dst = y + (static_cast<size_t>(tok) * a.H + h) * kP + 32 * half;
+                const int row0 = t_begin + b * kQ;
+                uint32_t w[16];
 #pragma unroll
-                    for (int c8 = 0; c8 < 4; ++c8) {
-                        uint32_t w[4];
+                for (int c = 0; c < 32; c += 2)
+                    w[c / 2] = pack_bf16(__uint_as_float(ya[c]) + et * __uint_as_float(ye[c]),
+                                         __uint_as_float(ya[c + 1]) + et * __uint_as_float(ye[c + 1]));
+                if (row0 + kQ <= t_end) {
+                    // whole block inside the sequence: stage the y tile in this block's X tile ((b) has read it) in
+                    // the layout of the tensor map and let one thread store it with TMA -- full 128-byte rows
+                    // instead of 32 scattered 16-byte pieces per warp instruction
+                    unsigned char *ys = sm + (b & 1) * kStageBytes;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int c = 8 * c8 + 2 * e;
-                            w[e] = pack_bf16(__uint_as_float(ya[c]) + et * __uint_as_float(ye[c]),
-                                             __uint_as_float(ya[c + 1]) + et * __uint_as_float(ye[c + 1]));
-                        }
-                        *reinterpret_cast<uint4 *>(dst + 8 * c8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (int c8 = 0; c8 < 4; ++c8)
+                        *reinterpret_cast<uint4 *>(ys + sw128_offset(t, 4 * half + c8)) = make_uint4(w[4 * c8], w[4 * c8 + 1], w[4 * c8 + 2], w[4 * c8 + 3]);
+                    fence_async_smem();
+                    named_bar_sync(2, 256);
+                    if (tid == 0) {
+                        tma_store_2d(&mapY, ys, h * kP, row0);
+                        tma_store_commit();
+                        tma_store_wait_read();
+                        mbar_arrive(&bars.x_free[b & 1]);
                     }
+                } else {
+                    const int tok = row0 + t;
+                    if (tok < t_end) {
+                        __nv_bfloat16 *dst = y + (static_cast<size_t>(tok) * a.H + h) * kP + 32 * half;
+#pragma unroll
+                        for (int c8 = 0; c8 < 4; ++c8)
+                            *reinterpret_cast<uint4 *>(dst + 8 * c8) = make_uint4(w[4 * c8], w[4 * c8 + 1], w[4 * c8 + 2], w[4 * c8 + 3]);
+                    }
+                    if (tid == 0) mbar_arrive(&bars.x_free[b & 1]);
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&bars.yo_done[b & 1]);
+            mbar_arrive(&bars.yo_done[b % 3]);
         }
     }
+    if (tid == 0) tma_store_wait_all();
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 13) tmem_dealloc(tm, kTmemCols);
+    if (warp == 17) tmem_dealloc(tm, kTmemCols);
 }
 
 }  // namespace
@@ -391,16 +446,17 @@ bool ssd_scan_tensor_supported(const SsdArgs &a, bool io_bf16) {
 }
 
 cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s) {
-    CUtensorMap mapX, mapB, mapC;
+    CUtensorMap mapX, mapB, mapC, mapY;
     const uint64_t rows = static_cast<uint64_t>(a.T_total);
     const uint64_t x_inner = static_cast<uint64_t>(a.H) * kP, bc_inner = static_cast<uint64_t>(a.G) * kN;
     if (!make_tensor_map_2d(&mapX, a.x, 2, x_inner, rows, x_inner * 2, 64, kQ, true) ||
         !make_tensor_map_2d(&mapB, a.B, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
-        !make_tensor_map_2d(&mapC, a.C, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true))
+        !make_tensor_map_2d(&mapC, a.C, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
+        !make_tensor_map_2d(&mapY, a.y, 2, x_inner, rows, x_inner * 2, 64, kQ, true))
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(ssd_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    ssd_scan_tensor_kernel<<<dim3(a.H, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapX, mapB, mapC);
+    ssd_scan_tensor_kernel<<<dim3(a.H, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapX, mapB, mapC, mapY);
     return cudaGetLastError();
 }
 
