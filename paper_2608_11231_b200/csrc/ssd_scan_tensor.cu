@@ -56,8 +56,7 @@ constexpr uint32_t kTmemCols = 512;
 struct Bars {
     uint64_t full_bc[2], full_x[2];                    // TMA transactions
     uint64_t bc_free[2], ac_done, y_done, h_done[2];   // tcgen05.commit targets
-    uint64_t x_free[2];                                // the epilogue thread that stores y out of the X tile
-    uint64_t mg_ready, yo_done[3];                     // 256 epilogue threads
+    uint64_t mg_ready, yo_done[3], ys_ready[2];        // 256 epilogue threads
     uint64_t sc_ready[3], x2_ready[2], hb_ready;       // 128 threads (scalar warps; hb_ready: state warps)
 };
 
@@ -98,9 +97,9 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
     if (tid == 0) {
         dead = 0;
         uint64_t *b1 = &bars.full_bc[0];
-        for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
+        for (int i = 0; i < 10; ++i) mbar_init(b1 + i, 1);
         uint64_t *b256 = &bars.mg_ready;
-        for (int i = 0; i < 4; ++i) mbar_init(b256 + i, 256);
+        for (int i = 0; i < 6; ++i) mbar_init(b256 + i, 256);
         uint64_t *b128 = &bars.sc_ready[0];
         for (int i = 0; i < 6; ++i) mbar_init(b128 + i, 128);
         mbar_fence_init();
@@ -119,21 +118,34 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             tma_prefetch_desc(&mapB);
             tma_prefetch_desc(&mapC);
             tma_prefetch_desc(&mapY);
-            for (int b = 0; b < nblk; ++b) {
-                // B and C of block b-2 are free after its (d); its X tile, which also stages y, after y has left it
+            for (int b = 0; b < nblk + 2; ++b) {
                 const int st = b & 1;
                 unsigned char *base = sm + st * kStageBytes;
                 const int row = t_begin + b * kQ;
-                if (b >= 2) mbar_wait(&bars.bc_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
-                mbar_expect_tx(&bars.full_bc[st], kBTile + kCTile);
-                for (int kb = 0; kb < 2; ++kb) {
-                    tma_load_2d(base + kXTile + kb * kQ * 128, &mapB, grp * kN + kb * 64, row, &bars.full_bc[st]);
-                    tma_load_2d(base + kXTile + kBTile + kb * kQ * 128, &mapC, grp * kN + kb * 64, row, &bars.full_bc[st]);
+                if (b < nblk) {
+                    // B and C of block b-2 are free after its (d)
+                    if (b >= 2) mbar_wait(&bars.bc_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                    mbar_expect_tx(&bars.full_bc[st], kBTile + kCTile);
+                    for (int kb = 0; kb < 2; ++kb) {
+                        tma_load_2d(base + kXTile + kb * kQ * 128, &mapB, grp * kN + kb * 64, row, &bars.full_bc[st]);
+                        tma_load_2d(base + kXTile + kBTile + kb * kQ * 128, &mapC, grp * kN + kb * 64, row, &bars.full_bc[st]);
+                    }
                 }
-                if (b >= 2) mbar_wait(&bars.x_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
-                mbar_expect_tx(&bars.full_x[st], kXTile);
-                tma_load_2d(base, &mapX, h * kP, row, &bars.full_x[st]);
+                if (b >= 2) {
+                    // the X tile of block b-2 now stages its y tile (whole blocks only): store it, then reuse the tile
+                    mbar_wait(&bars.ys_ready[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                    if (row - kQ <= t_end && !dead) {
+                        tma_store_2d(&mapY, base, h * kP, row - 2 * kQ);
+                        tma_store_commit();
+                        tma_store_wait_read();
+                    }
+                }
+                if (b < nblk) {
+                    mbar_expect_tx(&bars.full_x[st], kXTile);
+                    tma_load_2d(base, &mapX, h * kP, row, &bars.full_x[st]);
+                }
             }
+            tma_store_wait_all();
         }
     } else if (warp == 17) {
         // ======================================================= MMA issuer (one elected thread)
@@ -404,20 +416,13 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                                          __uint_as_float(ya[c + 1]) + et * __uint_as_float(ye[c + 1]));
                 if (row0 + kQ <= t_end) {
                     // whole block inside the sequence: stage the y tile in this block's X tile ((b) has read it) in
-                    // the layout of the tensor map and let one thread store it with TMA -- full 128-byte rows
+                    // the layout of the tensor map and let the TMA warp store it -- full 128-byte rows
                     // instead of 32 scattered 16-byte pieces per warp instruction
                     unsigned char *ys = sm + (b & 1) * kStageBytes;
 #pragma unroll
                     for (int c8 = 0; c8 < 4; ++c8)
                         *reinterpret_cast<uint4 *>(ys + sw128_offset(t, 4 * half + c8)) = make_uint4(w[4 * c8], w[4 * c8 + 1], w[4 * c8 + 2], w[4 * c8 + 3]);
                     fence_async_smem();
-                    named_bar_sync(2, 256);
-                    if (tid == 0) {
-                        tma_store_2d(&mapY, ys, h * kP, row0);
-                        tma_store_commit();
-                        tma_store_wait_read();
-                        mbar_arrive(&bars.x_free[b & 1]);
-                    }
                 } else {
                     const int tok = row0 + t;
                     if (tok < t_end) {
@@ -426,14 +431,13 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                         for (int c8 = 0; c8 < 4; ++c8)
                             *reinterpret_cast<uint4 *>(dst + 8 * c8) = make_uint4(w[4 * c8], w[4 * c8 + 1], w[4 * c8 + 2], w[4 * c8 + 3]);
                     }
-                    if (tid == 0) mbar_arrive(&bars.x_free[b & 1]);
                 }
+                mbar_arrive(&bars.ys_ready[b & 1]);
             }
             tc_fence_before_sync();
             mbar_arrive(&bars.yo_done[b % 3]);
         }
     }
-    if (tid == 0) tma_store_wait_all();
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 17) tmem_dealloc(tm, kTmemCols);

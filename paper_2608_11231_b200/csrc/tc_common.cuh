@@ -60,16 +60,29 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
 // Waits for the phase with the given parity.  `dead` is a CTA-wide flag in shared memory: once any
 // wait in the CTA has run out, every later wait returns at once, so a broken pipeline drains in
 // bounded time instead of spinning.  On timeout the device status word is set for the host to read.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status) {
-    if (mbar_test_wait(bar, parity)) return true;   // the common case in a pipeline that runs ahead
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *dead, int *status) {
     if (*dead) return false;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
         if ((it & 1023u) == 1023u && *dead) return false;
     }
     *dead = 1;
     if (status) atomicExch(status, 1);
     return false;
+}
+// The probe is inline (the common case in a pipeline that runs ahead); the polling loop is one shared
+// function so that the many waits of a warp-specialised kernel do not bloat its instruction footprint.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status) {
+    if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait_slow(smem_u32(bar), parity, dead, status);
 }
 
 // ------------------------------------------------------------------ TMA (tiled bulk tensor loads, 2-D)
