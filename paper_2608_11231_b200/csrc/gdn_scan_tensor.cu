@@ -21,7 +21,7 @@
 // (2) -> r -> (3) -> U o w -> (5) -> state copy.
 // A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
 // Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 out,
-// 12-15 prep, 16 TMA, 17 MMA issue.  All waits on mbarriers are bounded.
+// 12-15 prep, 16 TMA loads, 17 MMA issue, 18 TMA store of the output tile.  All waits on mbarriers are bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -33,7 +33,7 @@ using namespace tc;
 
 constexpr int kD = 128;   // d_k = d_v
 constexpr int kC = 64;    // tokens per block
-constexpr int kThreads = 576;
+constexpr int kThreads = 608;
 
 // shared-memory map (bytes, after 1024-byte alignment)
 constexpr int kQKStage = 4 * kC * 128;                 // [Q_kb0 | K_kb0 | Q_kb1 | K_kb1], each [64 rows x 128 B]
@@ -41,18 +41,19 @@ constexpr int kOffV = 2 * kQKStage;                    // V tile [64][128] bf16,
 constexpr int kOffSt = kOffV + kC * kD * 2;            // S^T bf16: [St_kb0 | St_kb1], each [128 rows x 128 B]
 constexpr int kOffR = kOffSt + 2 * kD * 128;           // R^T bf16 [128 rows x 128 B]
 constexpr int kOffUw = kOffR;                          // (U o w)^T bf16: written only after (3) has consumed R^T
-constexpr int kOffMPM = kOffR + kD * 128;              // [M; PM] bf16 [128 rows x 128 B], double-buffered
+constexpr int kOffMPM = kOffR + kD * 128;              // [M; PM] bf16 [128 rows x 128 B], double-buffered; once (3) has read it,
+                                                       // the buffer stages the block's output tile [64 tokens][128] bf16 for the TMA store
 constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] (A operand of (6); rows 64..127 unused)
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
 constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
 constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
 constexpr int kOffT = kOffM + kC * kLd * 4;            // block-product scratch, 3 x 16 x 16 fp32
-constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, double-buffered
+constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, three buffers
 constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxGroupRange = 100.f;                // log2 units: above this the per-group factors could overflow
-constexpr int kSmemBytes = kOffGb + 2 * kGbFloats * 4 + 1024;
-static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+constexpr int kSmemUsed = kOffGb + 3 * kGbFloats * 4;   // from the 1024-byte aligned base
+static_assert(kSmemUsed + 1024 <= 227 * 1024, "shared memory budget");
 
 // tensor-memory map (columns)
 constexpr uint32_t kTmG = 0;      // 64
@@ -64,9 +65,9 @@ constexpr uint32_t kTmemCols = 512;
 
 struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
-    uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done;
+    uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done, o_free[2];
     // 128-thread barriers (prep or out warpgroup)
-    uint64_t gb_ready[2], m_ready, mpm_ready[2], o_done[2], inv_done[2];
+    uint64_t gb_ready[3], m_ready, mpm_ready[2], o_done[2], inv_done[2], o_staged;
     // 64-thread barriers (the two halves of the out warpgroup)
     uint64_t a_ready, p_ready;
     // 256-thread barriers (both chain warpgroups)
@@ -96,7 +97,8 @@ __device__ __forceinline__ void store_row_chunks(unsigned char *tile, int row, i
 
 __global__ void __launch_bounds__(kThreads, 1)
 gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant__ CUtensorMap mapQ,
-                       const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV) {
+                       const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                       const __grid_constant__ CUtensorMap mapO) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ Bars bars;
@@ -106,6 +108,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, seq = blockIdx.y;
+    {
+        // the launch asks for all the dynamic shared memory the device has left; make sure the aligned map fits
+        uint32_t dyn;
+        asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+        if (static_cast<uint32_t>(sm - smem_raw) + kSmemUsed > dyn) {
+            if (tid == 0 && a.status) atomicExch(a.status, 1);
+            return;
+        }
+    }
     const int hk = h / (a.H_v / a.H_k);
     const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
     const int nblk = (t_end - t_begin + kC - 1) / kC;
@@ -119,9 +130,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     if (tid == 0) {
         dead = 0;
         uint64_t *b1 = &bars.full_qk[0];
-        for (int i = 0; i < 10; ++i) mbar_init(b1 + i, 1);
+        for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
         uint64_t *b128 = &bars.gb_ready[0];
-        for (int i = 0; i < 9; ++i) mbar_init(b128 + i, 128);
+        for (int i = 0; i < 11; ++i) mbar_init(b128 + i, 128);
         mbar_init(&bars.a_ready, 64);
         mbar_init(&bars.p_ready, 64);
         uint64_t *b256 = &bars.v_free;
@@ -156,6 +167,22 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
             }
         }
+    } else if (warp == 18) {
+        // ======================================================= TMA store of the output tiles (whole blocks only)
+        if (lane == 0) {
+            tma_prefetch_desc(&mapO);
+            for (int b = 0; b < nblk; ++b) {
+                mbar_wait(&bars.o_staged, b & 1, &dead, a.status);
+                const int t0 = t_begin + b * kC;
+                if (t0 + kC <= t_end && !dead) {
+                    tma_store_2d(&mapO, sm + kOffMPM + (b & 1) * (kD * 128), h * kD, t0);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+                mbar_arrive(&bars.o_free[b & 1]);
+            }
+            tma_store_wait_all();
+        }
     } else if (warp == 17) {
         // ======================================================= MMA issuer (one elected thread, tight code)
         if (elect_one()) {
@@ -186,10 +213,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.full_qk[0], 0, &dead, a.status);
             tc_fence_after_sync();
             issue_G(0);
-            mbar_wait(&bars.m_ready, 0, &dead, a.status);
-            mbar_wait(&bars.p_ready, 0, &dead, a.status);
-            tc_fence_after_sync();
-            issue_PM(0);
             for (int b = 0; b < nblk; ++b) {
                 const uint32_t par = b & 1;
                 const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
@@ -212,6 +235,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     tc_fence_after_sync();
                     issue_G(b + 1);
                 }
+                // (6) as soon as the inverse of this block is there; the prep warps turn it into the PM rows of the operand
+                mbar_wait(&bars.m_ready, par, &dead, a.status);
+                mbar_wait(&bars.p_ready, par, &dead, a.status);
+                tc_fence_after_sync();
+                issue_PM(b);
                 // (3) [U | PU] = R^T [M; PM]^T
                 mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
                 mbar_wait(&bars.r_ready, par, &dead, a.status);
@@ -228,13 +256,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmS, dUw + 2 * k, dKmn + ((k * 16 * 128) >> 4), idDS, true);
                 umma_commit(&bars.ds_done);
                 umma_commit(&bars.tiles_free_qk[b & 1]);
-                // (6) of the next block once its inverse is ready
-                if (b + 1 < nblk) {
-                    mbar_wait(&bars.m_ready, (b + 1) & 1, &dead, a.status);
-                    mbar_wait(&bars.p_ready, (b + 1) & 1, &dead, a.status);
-                    tc_fence_after_sync();
-                    issue_PM(b + 1);
-                }
             }
         }
     } else if (warp >= 12) {
@@ -253,14 +274,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         };
         float gv_next, bv_next;
         fetch_gb(0, gv_next, bv_next);
-        for (int b = 0; b < nblk; ++b) {
-            // buffers of parity b were last used by block b-2
-            if (b >= 2) {
-                mbar_wait(&bars.chain_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                mbar_wait(&bars.o_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-            }
+        auto prepare_scalars = [&](int b) {
             // ---- per-block scalars: cg, beta, gam = e^{cg}, w = e^{cg_C - cg}
-            float *sc = gb + (b & 1) * kGbFloats;
+            float *sc = gb + (b % 3) * kGbFloats;
             {
                 const float gv = gv_next, bv = bv_next;
                 fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
@@ -286,8 +302,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     if (x == 32) sc[5 * kC + 1] = bad ? 1.f : 0.f;
                 }
                 named_bar_sync(1, 128);
-                mbar_arrive(&bars.gb_ready[b & 1]);
+                mbar_arrive(&bars.gb_ready[b % 3]);
             }
+        };
+        prepare_scalars(0);
+        for (int b = 0; b < nblk; ++b) {
             // ---- P and A come from the out warpgroup (epilogue of (1))
             mbar_wait(&bars.a_ready, b & 1, &dead, a.status);
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
@@ -370,6 +389,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 named_bar_sync(1, 128);
             }
             // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
+            // the [M; PM] buffer of this parity was read by (3) of block b-2 and then staged that block's output tile
+            if (b >= 2) mbar_wait(&bars.o_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
             unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
             if (x < kC) {
                 const int t = x;
@@ -388,6 +409,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             fence_async_smem();
             mbar_arrive(&bars.m_ready);
             mbar_arrive(&bars.inv_done[b & 1]);
+            // ---- scalars of the next block, so that its mask epilogue runs while (6) of this one is in flight;
+            // their buffer was last read by the chain and the output epilogue of block b-2
+            if (b + 1 < nblk) {
+                if (b >= 2) {
+                    mbar_wait(&bars.chain_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+                    mbar_wait(&bars.o_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+                }
+                prepare_scalars(b + 1);
+            }
             // ---- PM rows (lanes 0..63 of the (6) accumulator) -> rows 64..127 of [M; PM]
             mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
@@ -416,8 +446,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         const int x = j;   // TMEM lane: 0..63 rows of Q K^T (-> P), 64..127 rows of K K^T (-> A)
         // epilogue of (1) for block b: P (bf16 operand of (6)) and A (fp32, input of the inverse)
         auto g_epilogue = [&](int b) {
-            const float *sc = gb + (b & 1) * kGbFloats;
-            mbar_wait(&bars.gb_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            const float *sc = gb + (b % 3) * kGbFloats;
+            mbar_wait(&bars.gb_ready[b % 3], (b / 3) & 1, &dead, a.status);
             float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
             if (x < kC) {
                 // the P buffer is free once (6) of block b-1 has read it
@@ -480,28 +510,49 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         g_epilogue(0);
         for (int b = 0; b < nblk; ++b) {
             if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
-            const float *sc = gb + (b & 1) * kGbFloats;
+            const float *sc = gb + (b % 3) * kGbFloats;
             mbar_wait(&bars.d1_done, b & 1, &dead, a.status);
             mbar_wait(&bars.up_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
             const int t0 = t_begin + b * kC;
             const int n = min(kC, t_end - t0);
-            __nv_bfloat16 *orow = o + (static_cast<size_t>(t0) * a.H_v + h) * kD + j;
+            if (n == kC) {
+                // whole block: stage the tile [token][j] in the [M; PM] buffer of this block, which (3) has finished
+                // reading (up_done); the store warp writes it out with TMA
+                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffMPM + (b & 1) * (kD * 128)) + j;
 #pragma unroll 1
-            for (int q = 0; q < 8; ++q) {
-                uint32_t qs[8], pu[8];
-                tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
-                tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
-                tmem_ld_wait();
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t qs[8], pu[8];
+                    tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
+                    tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
+                    tmem_ld_wait();
+                    const float4 g0 = *reinterpret_cast<const float4 *>(sc + 2 * kC + 8 * q);
+                    const float4 g1 = *reinterpret_cast<const float4 *>(sc + 2 * kC + 8 * q + 4);
+                    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int t = 8 * q + c;
-                    const float val = a.scale * fmaf(sc[2 * kC + t], __uint_as_float(qs[c]), __uint_as_float(pu[c]));
-                    if (t < n) orow[t * tstride] = __float2bfloat16_rn(val);
+                    for (int c = 0; c < 8; ++c)
+                        os[(8 * q + c) * kD] = __float2bfloat16_rn(a.scale * fmaf(gm[c], __uint_as_float(qs[c]), __uint_as_float(pu[c])));
+                }
+                fence_async_smem();
+            } else {
+                __nv_bfloat16 *orow = o + (static_cast<size_t>(t0) * a.H_v + h) * kD + j;
+#pragma unroll 1
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t qs[8], pu[8];
+                    tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
+                    tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int t = 8 * q + c;
+                        const float val = a.scale * fmaf(sc[2 * kC + t], __uint_as_float(qs[c]), __uint_as_float(pu[c]));
+                        if (t < n) orow[t * tstride] = __float2bfloat16_rn(val);
+                    }
                 }
             }
             tc_fence_before_sync();
             mbar_arrive(&bars.o_done[b & 1]);
+            mbar_arrive(&bars.o_staged);
         }
     } else {
         // ======================================================= chain warpgroups: lane = state column j, `half` = token / row half
@@ -530,9 +581,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         }
         for (int b = 0; b < nblk; ++b) {
             const uint32_t par = b & 1;
-            const float *sc = gb + (b & 1) * kGbFloats;
+            const float *sc = gb + (b % 3) * kGbFloats;
             const __nv_bfloat16 *vt = reinterpret_cast<const __nv_bfloat16 *>(sm + kOffV);
-            if (b > 0) mbar_wait(&bars.gb_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            if (b > 0) mbar_wait(&bars.gb_ready[b % 3], (b / 3) & 1, &dead, a.status);
             mbar_wait(&bars.full_v, par, &dead, a.status);
             mbar_wait(&bars.d1_done, par, &dead, a.status);
             tc_fence_after_sync();
@@ -576,8 +627,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const bool last = b + 1 == nblk;
             float gamN = 1.f;
             if (!last) {
-                mbar_wait(&bars.gb_ready[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
-                gamN = gb[((b + 1) & 1) * kGbFloats + 2 * kC + kC - 1];
+                mbar_wait(&bars.gb_ready[(b + 1) % 3], ((b + 1) / 3) & 1, &dead, a.status);
+                gamN = gb[((b + 1) % 3) * kGbFloats + 2 * kC + kC - 1];
             }
 #pragma unroll 1
             for (int q = 0; q < 4; ++q) {
@@ -622,16 +673,27 @@ bool gdn_scan_tensor_supported(const GdnArgs &a, bool io_bf16) {
 }
 
 cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s) {
-    CUtensorMap mapQ, mapK, mapV;
+    CUtensorMap mapQ, mapK, mapV, mapO;
     const uint64_t rows = static_cast<uint64_t>(a.T_total);
     const uint64_t qk_inner = static_cast<uint64_t>(a.H_k) * kD, v_inner = static_cast<uint64_t>(a.H_v) * kD;
     if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         !make_tensor_map_2d(&mapK, a.k, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
-        !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, kD, kC, false))
+        !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, kD, kC, false) ||
+        !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(gdn_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    // dynamic shared memory: everything the device allows beside the kernel's static part (the map needs
+    // kSmemUsed bytes from a 1024-byte aligned base; the kernel checks that it fits)
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, gdn_scan_tensor_kernel);
     if (e != cudaSuccess) return e;
-    gdn_scan_tensor_kernel<<<dim3(a.H_v, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapQ, mapK, mapV);
+    int dev = 0, optin = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+    const int dyn = optin - static_cast<int>(fa.sharedSizeBytes);
+    if (dyn < kSmemUsed) return cudaErrorInvalidConfiguration;
+    e = cudaFuncSetAttribute(gdn_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
+    if (e != cudaSuccess) return e;
+    gdn_scan_tensor_kernel<<<dim3(a.H_v, a.n_seq), kThreads, dyn, s>>>(a, mapQ, mapK, mapV, mapO);
     return cudaGetLastError();
 }
 
