@@ -7,8 +7,8 @@
 // gam_t = e^{cg_t}, Gam_ti = e^{cg_t - cg_i}, w_i = e^{cg_C - cg_i} and S the incoming state:
 //   (1) G    = [Q;K] K^T             rows 0..63: q_t.k_i, rows 64..127: k_t.k_i           tcgen05
 //       P_ti = Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)             out warps
-//       M    = (I + A)^{-1}          (UT transform: 16x16 diagonal blocks by substitution,
-//                                     off-diagonal blocks by block products, fp32)        prep warps
+//       M    = (I + A)^{-1}          (UT transform: 16x16 diagonal blocks by substitution in fp32,
+//                                     off-diagonal blocks by tf32 block products)         prep warps
 //   (6) PM   = P M                                                                        tcgen05
 //   (2) D1   = S^T [Q;K]^T           cols 0..63: (S^T q_t)_j, cols 64..127: (S^T k_t)_j    tcgen05
 //       r_t  = beta_t (v_t - gam_t S^T k_t)                                               chain warps
@@ -47,8 +47,7 @@ constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
 constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
 constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
-constexpr int kOffT = kOffM + kC * kLd * 4;            // block-product scratch, 3 x 16 x 16 fp32
-constexpr int kOffGb = kOffT + 3 * 256 * 4;            // per-block scalars, three buffers
+constexpr int kOffGb = kOffM + kC * kLd * 4;           // per-block scalars, three buffers
 constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxGroupRange = 100.f;                // log2 units: above this the per-group factors could overflow
@@ -74,6 +73,19 @@ struct Bars {
     uint64_t v_free, r_ready, uw_ready, st_ready, chain_done[2];
 };
 
+__device__ __forceinline__ uint32_t to_tf32(float v) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
+    return r;
+}
+// acc[16 x 8] += A[16 x 8] B[8 x 8] on the warp-level MMA; fragments as the PTX ISA lays them out
+// (row = lane / 4 (+8), column = lane % 4 (+4) for A; k = lane % 4 (+4), n = lane / 4 for B; row = lane / 4 (+8),
+// columns 2 (lane % 4), +1 for the accumulator).
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&acc)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ uint32_t elect_one() {
     uint32_t e;
@@ -263,7 +275,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         const int x = tid - 384;                 // 0..127 = TMEM lane
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         float *Mf = reinterpret_cast<float *>(sm + kOffM);
-        float *Tt = reinterpret_cast<float *>(sm + kOffT);
         auto fetch_gb = [&](int b, float &gv, float &bv) {
             const int t = t_begin + b * kC + x;
             gv = 0.f; bv = 0.f;
@@ -338,55 +349,45 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
             }
             named_bar_sync(1, 128);
-            // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc.
-            // A thread owns a 1 x 4 strip (row tt, columns 4*lg..4*lg+3) of a 16 x 16 block; operands are fetched
-            // eight k-steps at a time with 16-byte loads so that the loads of a group are in flight together.
-            for (int d = 1; d < 4; ++d) {
-                const int nstrip = (4 - d) * 64;
-                for (int e = x; e < nstrip; e += 128) {
-                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *arow = Af + (16 * r + tt) * kLd;
-                    const float *mcol = Mf + 16 * c + 4 * lg;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc, on the
+            // warp-level tensor-core MMA (m16n8k8, tf32 operands rounded to nearest, fp32 accumulation).  A unit is
+            // one 16 x 8 half of a block; its intermediate X = sum A_rm M_mc goes through the unused block (c, r)
+            // above the diagonal to change from accumulator to operand layout.
+            {
+                const int gid = lane >> 2, tig = lane & 3;
+                for (int d = 1; d < 4; ++d) {
+                    const int nunits = 2 * (4 - d);
+                    for (int u = warp & 3; u < nunits; u += 4) {
+                        const int c = u >> 1, nh = u & 1, r = c + d;
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-                    for (int ii = 16 * c; ii < 16 * r; ii += 8) {
-                        const float4 a0 = *reinterpret_cast<const float4 *>(arow + ii);
-                        const float4 a1 = *reinterpret_cast<const float4 *>(arow + ii + 4);
-                        float4 mv[8];
+                        for (int m = c; m < r; ++m) {
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) mv[u] = *reinterpret_cast<const float4 *>(mcol + (ii + u) * kLd);
-                        const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            acc.x = fmaf(av[u], mv[u].x, acc.x); acc.y = fmaf(av[u], mv[u].y, acc.y);
-                            acc.z = fmaf(av[u], mv[u].z, acc.z); acc.w = fmaf(av[u], mv[u].w, acc.w);
+                            for (int ks = 0; ks < 2; ++ks) {
+                                const float *ap = Af + (16 * r + gid) * kLd + 16 * m + 8 * ks + tig;
+                                const float *bp = Mf + (16 * m + 8 * ks + tig) * kLd + 16 * c + 8 * nh + gid;
+                                mma_tf32_16x8x8(acc, to_tf32(ap[0]), to_tf32(ap[8 * kLd]), to_tf32(ap[4]), to_tf32(ap[8 * kLd + 4]),
+                                                to_tf32(bp[0]), to_tf32(bp[4 * kLd]));
+                            }
                         }
-                    }
-                    *reinterpret_cast<float4 *>(Tt + c * 256 + tt * 16 + 4 * lg) = acc;
-                }
-                named_bar_sync(1, 128);
-                for (int e = x; e < nstrip; e += 128) {
-                    const int c = e >> 6, r = c + d, tt = (e >> 2) & 15, lg = e & 3;
-                    const float *drow = Mf + (16 * r + tt) * kLd + 16 * r;
-                    const float *tcol = Tt + c * 256 + 4 * lg;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                        float *xs = Mf + (16 * c) * kLd + 16 * r + 8 * nh;
+                        *reinterpret_cast<float2 *>(xs + gid * kLd + 2 * tig) = make_float2(acc[0], acc[1]);
+                        *reinterpret_cast<float2 *>(xs + (gid + 8) * kLd + 2 * tig) = make_float2(acc[2], acc[3]);
+                        __syncwarp();
+                        float out[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int i = 0; i < 16; i += 8) {
-                        const float4 d0 = *reinterpret_cast<const float4 *>(drow + i);
-                        const float4 d1 = *reinterpret_cast<const float4 *>(drow + i + 4);
-                        float4 tv[8];
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) tv[u] = *reinterpret_cast<const float4 *>(tcol + (i + u) * 16);
-                        const float dvv[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            acc.x = fmaf(dvv[u], tv[u].x, acc.x); acc.y = fmaf(dvv[u], tv[u].y, acc.y);
-                            acc.z = fmaf(dvv[u], tv[u].z, acc.z); acc.w = fmaf(dvv[u], tv[u].w, acc.w);
+                        for (int ks = 0; ks < 2; ++ks) {
+                            const float *dp = Mf + (16 * r + gid) * kLd + 16 * r + 8 * ks + tig;
+                            const float *xp = xs + (8 * ks + tig) * kLd + gid;
+                            mma_tf32_16x8x8(out, to_tf32(dp[0]), to_tf32(dp[8 * kLd]), to_tf32(dp[4]), to_tf32(dp[8 * kLd + 4]),
+                                            to_tf32(xp[0]), to_tf32(xp[4 * kLd]));
                         }
+                        float *mp = Mf + (16 * r + gid) * kLd + 16 * c + 8 * nh + 2 * tig;
+                        *reinterpret_cast<float2 *>(mp) = make_float2(-out[0], -out[1]);
+                        *reinterpret_cast<float2 *>(mp + 8 * kLd) = make_float2(-out[2], -out[3]);
                     }
-                    *reinterpret_cast<float4 *>(Mf + (16 * r + tt) * kLd + 16 * c + 4 * lg) = make_float4(-acc.x, -acc.y, -acc.z, -acc.w);
+                    named_bar_sync(1, 128);
                 }
-                named_bar_sync(1, 128);
             }
             // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
             // the [M; PM] buffer of this parity was read by (3) of block b-2 and then staged that block's output tile
