@@ -82,9 +82,69 @@ __device__ __forceinline__ uint32_t to_tf32(float v) {
 // (row = lane / 4 (+8), column = lane % 4 (+4) for A; k = lane % 4 (+4), n = lane / 4 for B; row = lane / 4 (+8),
 // columns 2 (lane % 4), +1 for the accumulator).
 __device__ __forceinline__ void mma_tf32_16x8x8(float (&acc)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// One off-diagonal block (r = c + D, c) of M = (I + A)^{-1}, or NH = 1 half of it (8 columns from 8 nh0):
+// X = sum_{m=c}^{r-1} A_rm M_mc, M_rc = -D_r X with D_r the inverted diagonal block.  tf32 operands rounded to
+// nearest, fp32 accumulation.  Every MMA of a stage has its own accumulator, so they are all in flight together
+// (the warp-level MMA has a long latency here); X passes through the unused block (c, r) above the diagonal to
+// change from accumulator to operand layout.  A, M: fp32 [64][ld].
+template <int NH, int D>
+__device__ __forceinline__ void inv_offdiag(const float *Af, float *Mf, int c, int nh0, int gid, int tig) {
+    constexpr int ld = kLd;
+    const int r = c + D;
+    float part[D][2][NH][4];
+#pragma unroll
+    for (int mm = 0; mm < D; ++mm) {
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+            const float *ap = Af + (16 * r + gid) * ld + 16 * (c + mm) + 8 * ks + tig;
+            const uint32_t a0 = to_tf32(ap[0]), a1 = to_tf32(ap[8 * ld]), a2 = to_tf32(ap[4]), a3 = to_tf32(ap[8 * ld + 4]);
+#pragma unroll
+            for (int hh = 0; hh < NH; ++hh) {
+                const float *bp = Mf + (16 * (c + mm) + 8 * ks + tig) * ld + 16 * c + 8 * (nh0 + hh) + gid;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) part[mm][ks][hh][i] = 0.f;
+                mma_tf32_16x8x8(part[mm][ks][hh], a0, a1, a2, a3, to_tf32(bp[0]), to_tf32(bp[4 * ld]));
+            }
+        }
+    }
+    float *xs = Mf + (16 * c) * ld + 16 * r + 8 * nh0;
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int mm = 0; mm < D; ++mm)
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) x[i] += part[mm][ks][hh][i];
+        *reinterpret_cast<float2 *>(xs + 8 * hh + gid * ld + 2 * tig) = make_float2(x[0], x[1]);
+        *reinterpret_cast<float2 *>(xs + 8 * hh + (gid + 8) * ld + 2 * tig) = make_float2(x[2], x[3]);
+    }
+    __syncwarp();
+    float out[2][NH][4];
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+        const float *dp = Mf + (16 * r + gid) * ld + 16 * r + 8 * ks + tig;
+        const uint32_t a0 = to_tf32(dp[0]), a1 = to_tf32(dp[8 * ld]), a2 = to_tf32(dp[4]), a3 = to_tf32(dp[8 * ld + 4]);
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) {
+            const float *xp = xs + 8 * hh + (8 * ks + tig) * ld + gid;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) out[ks][hh][i] = 0.f;
+            mma_tf32_16x8x8(out[ks][hh], a0, a1, a2, a3, to_tf32(xp[0]), to_tf32(xp[4 * ld]));
+        }
+    }
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+        float *mp = Mf + (16 * r + gid) * ld + 16 * c + 8 * (nh0 + hh) + 2 * tig;
+        *reinterpret_cast<float2 *>(mp) = make_float2(-(out[0][hh][0] + out[1][hh][0]), -(out[0][hh][1] + out[1][hh][1]));
+        *reinterpret_cast<float2 *>(mp + 8 * ld) = make_float2(-(out[0][hh][2] + out[1][hh][2]), -(out[0][hh][3] + out[1][hh][3]));
+    }
 }
 __device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ uint32_t elect_one() {
@@ -349,45 +409,16 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
             }
             named_bar_sync(1, 128);
-            // Off-diagonal blocks by distance d from the diagonal: M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc, on the
-            // warp-level tensor-core MMA (m16n8k8, tf32 operands rounded to nearest, fp32 accumulation).  A unit is
-            // one 16 x 8 half of a block; its intermediate X = sum A_rm M_mc goes through the unused block (c, r)
-            // above the diagonal to change from accumulator to operand layout.
+            // Off-diagonal blocks by distance d from the diagonal, M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc, on the
+            // warp-level tensor-core MMA; one warp per block (d = 1) or half block (d = 2, 3).
             {
-                const int gid = lane >> 2, tig = lane & 3;
-                for (int d = 1; d < 4; ++d) {
-                    const int nunits = 2 * (4 - d);
-                    for (int u = warp & 3; u < nunits; u += 4) {
-                        const int c = u >> 1, nh = u & 1, r = c + d;
-                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-                        for (int m = c; m < r; ++m) {
-#pragma unroll
-                            for (int ks = 0; ks < 2; ++ks) {
-                                const float *ap = Af + (16 * r + gid) * kLd + 16 * m + 8 * ks + tig;
-                                const float *bp = Mf + (16 * m + 8 * ks + tig) * kLd + 16 * c + 8 * nh + gid;
-                                mma_tf32_16x8x8(acc, to_tf32(ap[0]), to_tf32(ap[8 * kLd]), to_tf32(ap[4]), to_tf32(ap[8 * kLd + 4]),
-                                                to_tf32(bp[0]), to_tf32(bp[4 * kLd]));
-                            }
-                        }
-                        float *xs = Mf + (16 * c) * kLd + 16 * r + 8 * nh;
-                        *reinterpret_cast<float2 *>(xs + gid * kLd + 2 * tig) = make_float2(acc[0], acc[1]);
-                        *reinterpret_cast<float2 *>(xs + (gid + 8) * kLd + 2 * tig) = make_float2(acc[2], acc[3]);
-                        __syncwarp();
-                        float out[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                        for (int ks = 0; ks < 2; ++ks) {
-                            const float *dp = Mf + (16 * r + gid) * kLd + 16 * r + 8 * ks + tig;
-                            const float *xp = xs + (8 * ks + tig) * kLd + gid;
-                            mma_tf32_16x8x8(out, to_tf32(dp[0]), to_tf32(dp[8 * kLd]), to_tf32(dp[4]), to_tf32(dp[8 * kLd + 4]),
-                                            to_tf32(xp[0]), to_tf32(xp[4 * kLd]));
-                        }
-                        float *mp = Mf + (16 * r + gid) * kLd + 16 * c + 8 * nh + 2 * tig;
-                        *reinterpret_cast<float2 *>(mp) = make_float2(-out[0], -out[1]);
-                        *reinterpret_cast<float2 *>(mp + 8 * kLd) = make_float2(-out[2], -out[3]);
-                    }
-                    named_bar_sync(1, 128);
-                }
+                const int wq = warp & 3, gid = lane >> 2, tig = lane & 3;
+                if (wq < 3) inv_offdiag<2, 1>(Af, Mf, wq, 0, gid, tig);
+                named_bar_sync(1, 128);
+                inv_offdiag<1, 2>(Af, Mf, wq >> 1, wq & 1, gid, tig);
+                named_bar_sync(1, 128);
+                if (wq < 2) inv_offdiag<1, 3>(Af, Mf, 0, wq, gid, tig);
+                named_bar_sync(1, 128);
             }
             // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
             // the [M; PM] buffer of this parity was read by (3) of block b-2 and then staged that block's output tile
