@@ -47,11 +47,11 @@ constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
 constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
 constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
-constexpr int kOffGb = kOffM + kC * kLd * 4;           // per-block scalars, three buffers
+constexpr int kOffGb = kOffM + kC * kLd * 4;           // per-block scalars, four buffers (prepared two blocks ahead)
 constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxGroupRange = 100.f;                // log2 units: above this the per-group factors could overflow
-constexpr int kSmemUsed = kOffGb + 3 * kGbFloats * 4;   // from the 1024-byte aligned base
+constexpr int kSmemUsed = kOffGb + 4 * kGbFloats * 4;   // from the 1024-byte aligned base
 static_assert(kSmemUsed + 1024 <= 227 * 1024, "shared memory budget");
 
 // tensor-memory map (columns)
@@ -66,7 +66,7 @@ struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
     uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done, o_free[2];
     // 128-thread barriers (prep or out warpgroup)
-    uint64_t gb_ready[3], m_ready, mpm_ready[2], o_done[2], inv_done[2], o_staged;
+    uint64_t gb_ready[4], m_ready, mpm_ready[2], o_done[2], inv_done[2], o_staged;
     // 64-thread barriers (the two halves of the out warpgroup)
     uint64_t a_ready, p_ready;
     // 256-thread barriers (both chain warpgroups)
@@ -204,7 +204,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         uint64_t *b1 = &bars.full_qk[0];
         for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
         uint64_t *b128 = &bars.gb_ready[0];
-        for (int i = 0; i < 11; ++i) mbar_init(b128 + i, 128);
+        for (int i = 0; i < 12; ++i) mbar_init(b128 + i, 128);
         mbar_init(&bars.a_ready, 64);
         mbar_init(&bars.p_ready, 64);
         uint64_t *b256 = &bars.v_free;
@@ -347,7 +347,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         fetch_gb(0, gv_next, bv_next);
         auto prepare_scalars = [&](int b) {
             // ---- per-block scalars: cg, beta, gam = e^{cg}, w = e^{cg_C - cg}
-            float *sc = gb + (b % 3) * kGbFloats;
+            float *sc = gb + (b & 3) * kGbFloats;
             {
                 const float gv = gv_next, bv = bv_next;
                 fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
@@ -373,13 +373,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     if (x == 32) sc[5 * kC + 1] = bad ? 1.f : 0.f;
                 }
                 named_bar_sync(1, 128);
-                mbar_arrive(&bars.gb_ready[b % 3]);
+                mbar_arrive(&bars.gb_ready[b & 3]);
             }
         };
         prepare_scalars(0);
+        if (nblk > 1) prepare_scalars(1);
         for (int b = 0; b < nblk; ++b) {
             // ---- P and A come from the out warpgroup (epilogue of (1))
             mbar_wait(&bars.a_ready, b & 1, &dead, a.status);
+            named_bar_sync(1, 128);   // every thread is done with the fp32 M of the previous block
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
             // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k by forward
             // substitution; each row of the block is fetched with four 16-byte loads ahead of its use.
@@ -441,14 +443,14 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             fence_async_smem();
             mbar_arrive(&bars.m_ready);
             mbar_arrive(&bars.inv_done[b & 1]);
-            // ---- scalars of the next block, so that its mask epilogue runs while (6) of this one is in flight;
-            // their buffer was last read by the chain and the output epilogue of block b-2
-            if (b + 1 < nblk) {
+            // ---- scalars of block b+2 while (6) of this one is in flight, so that the mask epilogue of the next
+            // block never waits for them; their buffer was last read by the chain and the output epilogue of block b-2
+            if (b + 2 < nblk) {
                 if (b >= 2) {
                     mbar_wait(&bars.chain_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
                     mbar_wait(&bars.o_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
                 }
-                prepare_scalars(b + 1);
+                prepare_scalars(b + 2);
             }
             // ---- PM rows (lanes 0..63 of the (6) accumulator) -> rows 64..127 of [M; PM]
             mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
@@ -478,8 +480,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         const int x = j;   // TMEM lane: 0..63 rows of Q K^T (-> P), 64..127 rows of K K^T (-> A)
         // epilogue of (1) for block b: P (bf16 operand of (6)) and A (fp32, input of the inverse)
         auto g_epilogue = [&](int b) {
-            const float *sc = gb + (b % 3) * kGbFloats;
-            mbar_wait(&bars.gb_ready[b % 3], (b / 3) & 1, &dead, a.status);
+            const float *sc = gb + (b & 3) * kGbFloats;
+            mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
             float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
             if (x < kC) {
                 // the P buffer is free once (6) of block b-1 has read it
@@ -542,7 +544,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         g_epilogue(0);
         for (int b = 0; b < nblk; ++b) {
             if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
-            const float *sc = gb + (b % 3) * kGbFloats;
+            const float *sc = gb + (b & 3) * kGbFloats;
             mbar_wait(&bars.d1_done, b & 1, &dead, a.status);
             mbar_wait(&bars.up_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
@@ -613,9 +615,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         }
         for (int b = 0; b < nblk; ++b) {
             const uint32_t par = b & 1;
-            const float *sc = gb + (b % 3) * kGbFloats;
+            const float *sc = gb + (b & 3) * kGbFloats;
             const __nv_bfloat16 *vt = reinterpret_cast<const __nv_bfloat16 *>(sm + kOffV);
-            if (b > 0) mbar_wait(&bars.gb_ready[b % 3], (b / 3) & 1, &dead, a.status);
+            if (b > 0) mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
             mbar_wait(&bars.full_v, par, &dead, a.status);
             mbar_wait(&bars.d1_done, par, &dead, a.status);
             tc_fence_after_sync();
@@ -659,8 +661,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const bool last = b + 1 == nblk;
             float gamN = 1.f;
             if (!last) {
-                mbar_wait(&bars.gb_ready[(b + 1) % 3], ((b + 1) / 3) & 1, &dead, a.status);
-                gamN = gb[((b + 1) % 3) * kGbFloats + 2 * kC + kC - 1];
+                mbar_wait(&bars.gb_ready[(b + 1) & 3], ((b + 1) >> 2) & 1, &dead, a.status);
+                gamN = gb[((b + 1) & 3) * kGbFloats + 2 * kC + kC - 1];
             }
 #pragma unroll 1
             for (int q = 0; q < 4; ++q) {
