@@ -21,7 +21,8 @@
 // (2) -> r -> (3) -> U o w -> (5) -> state copy.
 // A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
 // Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 out,
-// 12-15 prep, 16 TMA loads, 17 MMA issue, 18 TMA store of the output tile.  All waits on mbarriers are bounded.
+// 12-15 prep (the inverse), 16 TMA loads, 17 MMA issue, 18 TMA store of the output tile, 19 per-block scalars
+// (running up to three blocks ahead).  All waits on mbarriers are bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -33,7 +34,7 @@ using namespace tc;
 
 constexpr int kD = 128;   // d_k = d_v
 constexpr int kC = 64;    // tokens per block
-constexpr int kThreads = 608;
+constexpr int kThreads = 640;
 
 // shared-memory map (bytes, after 1024-byte alignment)
 constexpr int kQKStage = 4 * kC * 128;                 // [Q_kb0 | K_kb0 | Q_kb1 | K_kb1], each [64 rows x 128 B]
@@ -43,7 +44,8 @@ constexpr int kOffR = kOffSt + 2 * kD * 128;           // R^T bf16 [128 rows x 1
 constexpr int kOffUw = kOffR;                          // (U o w)^T bf16: written only after (3) has consumed R^T
 constexpr int kOffMPM = kOffR + kD * 128;              // [M; PM] bf16 [128 rows x 128 B], double-buffered; once (3) has read it,
                                                        // the buffer stages the block's output tile [64 tokens][128] bf16 for the TMA store
-constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] (A operand of (6); rows 64..127 unused)
+constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] = rows 64..127 of the A operand of (6), whose rows
+                                                       // 0..63 (the end of the [M; PM] buffers) are don't-care: PM lands in TMEM lanes 64..127
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
 constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
 constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
@@ -66,11 +68,11 @@ struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
     uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done, o_free[2];
     // 128-thread barriers (prep or out warpgroup)
-    uint64_t gb_ready[4], m_ready, mpm_ready[2], o_done[2], inv_done[2], o_staged;
+    uint64_t m_ready[2], o_done[4], inv_done[2], o_staged;
     // 64-thread barriers (the two halves of the out warpgroup)
-    uint64_t a_ready, p_ready;
+    uint64_t a_ready, p_ready, gb_ready[4], mpm_ready[2];
     // 256-thread barriers (both chain warpgroups)
-    uint64_t v_free, r_ready, uw_ready, st_ready, chain_done[2];
+    uint64_t v_free, r_ready, uw_ready, st_ready, chain_done[4];
 };
 
 __device__ __forceinline__ uint32_t to_tf32(float v) {
@@ -176,7 +178,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     __shared__ Bars bars;
     __shared__ uint32_t tmem_base;
     __shared__ int dead;
-    __shared__ float scan_carry;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, seq = blockIdx.y;
@@ -203,12 +204,12 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         dead = 0;
         uint64_t *b1 = &bars.full_qk[0];
         for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
-        uint64_t *b128 = &bars.gb_ready[0];
-        for (int i = 0; i < 12; ++i) mbar_init(b128 + i, 128);
-        mbar_init(&bars.a_ready, 64);
-        mbar_init(&bars.p_ready, 64);
+        uint64_t *b128 = &bars.m_ready[0];
+        for (int i = 0; i < 9; ++i) mbar_init(b128 + i, 128);
+        uint64_t *b64 = &bars.a_ready;
+        for (int i = 0; i < 8; ++i) mbar_init(b64 + i, (i >= 2 && i < 6) ? 32 : 64);   // gb_ready: the scalar warp
         uint64_t *b256 = &bars.v_free;
-        for (int i = 0; i < 6; ++i) mbar_init(b256 + i, 256);
+        for (int i = 0; i < 8; ++i) mbar_init(b256 + i, 256);
         mbar_fence_init();
     }
     if (warp == 17) tmem_alloc(&tmem_base, kTmemCols);
@@ -227,6 +228,14 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             for (int b = 0; b < nblk; ++b) {
                 const int st = b & 1;
                 const int row = t_begin + b * kC;
+                // the two-stage ring cannot hide the DRAM latency of the tile loads: pull the tiles of block b+2 into L2 now
+                if (b + 2 < nblk) {
+                    for (int kb = 0; kb < 2; ++kb) {
+                        tma_prefetch_l2_2d(&mapQ, hk * kD + kb * 64, row + 2 * kC);
+                        tma_prefetch_l2_2d(&mapK, hk * kD + kb * 64, row + 2 * kC);
+                    }
+                    tma_prefetch_l2_2d(&mapV, h * kD, row + 2 * kC);
+                }
                 if (b >= 2) mbar_wait(&bars.tiles_free_qk[st], ((b - 2) >> 1) & 1, &dead, a.status);
                 unsigned char *base = sm + st * kQKStage;
                 mbar_expect_tx(&bars.full_qk[st], kQKStage);
@@ -238,6 +247,55 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 mbar_expect_tx(&bars.full_v, kC * kD * 2);
                 tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
             }
+        }
+    } else if (warp == 19) {
+        // ======================================================= scalar warp: lane = tokens 2 lane, 2 lane + 1 of the block
+        auto fetch_gb = [&](int b, float2 &gv, float2 &bv) {
+            const int t = t_begin + b * kC + 2 * lane;
+            gv = make_float2(0.f, 0.f); bv = make_float2(0.f, 0.f);
+            if (b < nblk && t < t_end) {
+                gv.x = a.g[static_cast<size_t>(t) * a.H_v + h];
+                bv.x = a.beta[static_cast<size_t>(t) * a.H_v + h];
+            }
+            if (b < nblk && t + 1 < t_end) {
+                gv.y = a.g[static_cast<size_t>(t + 1) * a.H_v + h];
+                bv.y = a.beta[static_cast<size_t>(t + 1) * a.H_v + h];
+            }
+        };
+        float2 gv_next, bv_next;
+        fetch_gb(0, gv_next, bv_next);
+        for (int b = 0; b < nblk; ++b) {
+            // the buffer of block b was last read by the chain and the output epilogue of block b-4
+            if (b >= 4) {
+                mbar_wait(&bars.chain_done[b & 3], ((b - 4) >> 2) & 1, &dead, a.status);
+                mbar_wait(&bars.o_done[b & 3], ((b - 4) >> 2) & 1, &dead, a.status);
+            }
+            // ---- per-block scalars: cg (in log2 units), beta, gam = e^{cg}, w = e^{cg_C - cg}, group factors
+            float *sc = gb + (b & 3) * kGbFloats;
+            const float2 gv = gv_next, bv = bv_next;
+            fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
+            const float pair = gv.x + gv.y;
+            float run = pair;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float up = __shfl_up_sync(0xffffffffu, run, o);
+                if (lane >= o) run += up;
+            }
+            const float c0 = (run - gv.y) * kLog2e, c1 = run * kLog2e;
+            const float last = __shfl_sync(0xffffffffu, c1, 31);
+            // first column of each group of 16 tokens = first token of lanes 0, 8, 16, 24
+            const float ref = __shfl_sync(0xffffffffu, c0, lane & ~7);
+            const float r0 = ref - c0, r1 = ref - c1;
+            const int t = 2 * lane;
+            *reinterpret_cast<float2 *>(sc + t) = make_float2(c0, c1);
+            *reinterpret_cast<float2 *>(sc + kC + t) = bv;
+            *reinterpret_cast<float2 *>(sc + 2 * kC + t) = make_float2(exp2f(c0), exp2f(c1));
+            *reinterpret_cast<float2 *>(sc + 3 * kC + t) = make_float2(exp2f(last - c0), exp2f(last - c1));
+            // factor of a column relative to the first column of its group (>= 1)
+            *reinterpret_cast<float2 *>(sc + 4 * kC + t) = make_float2(exp2f(fminf(r0, 126.f)), exp2f(fminf(r1, 126.f)));
+            const unsigned bad = __ballot_sync(0xffffffffu, r0 > kMaxGroupRange || r1 > kMaxGroupRange);
+            if (lane == 0) *reinterpret_cast<float2 *>(sc + 5 * kC) = make_float2(bad ? 1.f : 0.f, 0.f);
+            mbar_arrive(&bars.gb_ready[b & 3]);
         }
     } else if (warp == 18) {
         // ======================================================= TMA store of the output tiles (whole blocks only)
@@ -265,7 +323,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const uint64_t dSt = umma_desc(smem_u32(sm + kOffSt), 0, 1024);
             const uint64_t dR = umma_desc(smem_u32(sm + kOffR), 0, 1024);
             const uint64_t dUw = umma_desc(smem_u32(sm + kOffUw), 0, 1024);
-            const uint64_t dP = umma_desc(smem_u32(sm + kOffP), 0, 1024);
+            const uint64_t dP = umma_desc(smem_u32(sm + kOffP - kC * 128), 0, 1024);
             const uint64_t dMPM0 = umma_desc(smem_u32(sm + kOffMPM), 0, 1024);
             auto issue_G = [&](int b) {
                 const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
@@ -288,30 +346,41 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             for (int b = 0; b < nblk; ++b) {
                 const uint32_t par = b & 1;
                 const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
-                // (2) needs the bf16 state copy of block b and the D1 / UP accumulators drained
-                mbar_wait(&bars.st_ready, par, &dead, a.status);
-                if (b > 0) mbar_wait(&bars.o_done[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
-                tc_fence_after_sync();
+                // Three MMAs of this iteration have independent inputs and are issued in the order their inputs arrive
+                // (a blocking wait for one would hold back the others):
+                //   (6) of block b:   the inverse (m_ready) and P (p_ready);
+                //   (2) of block b:   the bf16 state copy (st_ready) and the D1 / UP accumulators drained (o_done of b-1);
+                //   (1) of block b+1: the G columns drained by the mask epilogue of block b, and the next Q / K tiles.
+                uint32_t pending = 4u | 1u | (b + 1 < nblk ? 2u : 0u);
+                for (uint32_t spins = 0; pending != 0;) {
+                    if ((pending & 4u) && mbar_test_wait(&bars.m_ready[b & 1], (b >> 1) & 1) && mbar_test_wait(&bars.p_ready, par)) {
+                        tc_fence_after_sync();
+                        issue_PM(b);
+                        pending &= ~4u;
+                    } else if ((pending & 1u) && mbar_test_wait(&bars.st_ready, par) &&
+                               (b == 0 || mbar_test_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1))) {
+                        tc_fence_after_sync();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint64_t offA = ((k >> 2) * (kD * 128) + (k & 3) * 32) >> 4;
-                    const uint64_t offB = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
-                    umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
+                        for (int k = 0; k < 8; ++k) {
+                            const uint64_t offA = ((k >> 2) * (kD * 128) + (k & 3) * 32) >> 4;
+                            const uint64_t offB = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
+                            umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
+                        }
+                        umma_commit(&bars.d1_done);
+                        pending &= ~1u;
+                    } else if ((pending & 2u) && mbar_test_wait(&bars.a_ready, par) && mbar_test_wait(&bars.p_ready, par) &&
+                               mbar_test_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1)) {
+                        tc_fence_after_sync();
+                        issue_G(b + 1);
+                        pending &= ~2u;
+                    } else if (++spins > kSpinLimit || dead) {
+                        if (!dead) {
+                            dead = 1;
+                            if (a.status) atomicExch(a.status, 1);
+                        }
+                        break;
+                    }
                 }
-                umma_commit(&bars.d1_done);
-                // (1) of the next block right behind (2), as soon as the epilogue of block b has drained the G columns
-                if (b + 1 < nblk) {
-                    mbar_wait(&bars.a_ready, par, &dead, a.status);
-                    mbar_wait(&bars.p_ready, par, &dead, a.status);
-                    mbar_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
-                    tc_fence_after_sync();
-                    issue_G(b + 1);
-                }
-                // (6) as soon as the inverse of this block is there; the prep warps turn it into the PM rows of the operand
-                mbar_wait(&bars.m_ready, par, &dead, a.status);
-                mbar_wait(&bars.p_ready, par, &dead, a.status);
-                tc_fence_after_sync();
-                issue_PM(b);
                 // (3) [U | PU] = R^T [M; PM]^T
                 mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
                 mbar_wait(&bars.r_ready, par, &dead, a.status);
@@ -331,53 +400,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             }
         }
     } else if (warp >= 12) {
-        // ======================================================= prep warpgroup (one block ahead)
-        const int x = tid - 384;                 // 0..127 = TMEM lane
-        const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        // ======================================================= prep warpgroup: the inverse, ahead of the chain
+        const int x = tid - 384;                 // 0..127
         float *Mf = reinterpret_cast<float *>(sm + kOffM);
-        auto fetch_gb = [&](int b, float &gv, float &bv) {
-            const int t = t_begin + b * kC + x;
-            gv = 0.f; bv = 0.f;
-            if (x < kC && b < nblk && t < t_end) {
-                gv = a.g[static_cast<size_t>(t) * a.H_v + h];
-                bv = a.beta[static_cast<size_t>(t) * a.H_v + h];
-            }
-        };
-        float gv_next, bv_next;
-        fetch_gb(0, gv_next, bv_next);
-        auto prepare_scalars = [&](int b) {
-            // ---- per-block scalars: cg, beta, gam = e^{cg}, w = e^{cg_C - cg}
-            float *sc = gb + (b & 3) * kGbFloats;
-            {
-                const float gv = gv_next, bv = bv_next;
-                fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
-                float run = gv;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float up = __shfl_up_sync(0xffffffffu, run, o);
-                    if (lane >= o) run += up;
-                }
-                if (x == 31) scan_carry = run;
-                named_bar_sync(1, 128);
-                if (x >= 32 && x < kC) run += scan_carry;
-                const float c2 = run * kLog2e;
-                if (x < kC) { sc[x] = c2; sc[kC + x] = bv; sc[2 * kC + x] = exp2f(c2); }
-                named_bar_sync(1, 128);
-                if (x < kC) {
-                    sc[3 * kC + x] = exp2f(sc[kC - 1] - c2);
-                    // factor of column x relative to the first column of its group of 16 (>= 1)
-                    const float rng = sc[x & ~15] - c2;
-                    sc[4 * kC + x] = exp2f(fminf(rng, 126.f));
-                    const unsigned bad = __ballot_sync(0xffffffffu, rng > kMaxGroupRange);
-                    if (x == 0) sc[5 * kC] = bad ? 1.f : 0.f;
-                    if (x == 32) sc[5 * kC + 1] = bad ? 1.f : 0.f;
-                }
-                named_bar_sync(1, 128);
-                mbar_arrive(&bars.gb_ready[b & 3]);
-            }
-        };
-        prepare_scalars(0);
-        if (nblk > 1) prepare_scalars(1);
         for (int b = 0; b < nblk; ++b) {
             // ---- P and A come from the out warpgroup (epilogue of (1))
             mbar_wait(&bars.a_ready, b & 1, &dead, a.status);
@@ -426,10 +451,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             // the [M; PM] buffer of this parity was read by (3) of block b-2 and then staged that block's output tile
             if (b >= 2) mbar_wait(&bars.o_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
             unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
-            if (x < kC) {
-                const int t = x;
-#pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
+            {
+                // thread = (row t, half of the columns)
+                const int t = x & 63, q0 = 2 * (x >> 6);
+#pragma unroll
+                for (int q = q0; q < q0 + 2; ++q) {
                     float v[16];
 #pragma unroll
                     for (int c = 0; c < 16; c += 4) {
@@ -441,35 +467,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
             }
             fence_async_smem();
-            mbar_arrive(&bars.m_ready);
+            mbar_arrive(&bars.m_ready[b & 1]);
             mbar_arrive(&bars.inv_done[b & 1]);
-            // ---- scalars of block b+2 while (6) of this one is in flight, so that the mask epilogue of the next
-            // block never waits for them; their buffer was last read by the chain and the output epilogue of block b-2
-            if (b + 2 < nblk) {
-                if (b >= 2) {
-                    mbar_wait(&bars.chain_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                    mbar_wait(&bars.o_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                }
-                prepare_scalars(b + 2);
-            }
-            // ---- PM rows (lanes 0..63 of the (6) accumulator) -> rows 64..127 of [M; PM]
-            mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            if (x < kC) {
-#pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t rr[16];
-                    tmem_ld16(lane_base + kTmPM + 16 * q, rr);
-                    tmem_ld_wait();
-                    float v[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
-                    store_row_chunks(mpm, kC + x, 2 * q, v);
-                }
-            }
-            fence_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&bars.mpm_ready[b & 1]);
         }
     } else if (warp >= 8) {
         // ======================================================= out warpgroup: o_t[j] = scale (gam_t (S^T q_t)_j + (P u)_t[j]); lane = j
@@ -479,16 +478,42 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         const size_t tstride = static_cast<size_t>(a.H_v) * kD;
         const int x = j;   // TMEM lane: 0..63 rows of Q K^T (-> P), 64..127 rows of K K^T (-> A)
         // epilogue of (1) for block b: P (bf16 operand of (6)) and A (fp32, input of the inverse)
+        // PM rows of block b (lanes 64..127 of the (6) accumulator) -> rows 64..127 of [M; PM]; warps 10 and 11 only,
+        // so that the P rows of the next block (warps 8 and 9) are worked on at the same time
+        auto pm_rows = [&](int b) {
+            mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
+#pragma unroll 1
+            for (int q = 0; q < 4; ++q) {
+                uint32_t rr[16];
+                tmem_ld16(lane_base + kTmPM + 16 * q, rr);
+                tmem_ld_wait();
+                float v[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
+                store_row_chunks(mpm, x, 2 * q, v);
+            }
+            fence_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&bars.mpm_ready[b & 1]);
+        };
         auto g_epilogue = [&](int b) {
             const float *sc = gb + (b & 3) * kGbFloats;
             mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
             float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
+            bool pm_pending = x >= kC && b >= 1;
             if (x < kC) {
                 // the P buffer is free once (6) of block b-1 has read it
                 if (b >= 1) mbar_wait(&bars.pm_done, (b - 1) & 1, &dead, a.status);
             } else {
                 // the A buffer of this parity is free once block b-2 has been inverted
                 if (b >= 2) mbar_wait(&bars.inv_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+                // the result of (6) of block b-1 is on the chain's critical path: take it first if it is there already
+                if (pm_pending && __all_sync(0xffffffffu, mbar_test_wait(&bars.pm_done, (b - 1) & 1))) {
+                    pm_rows(b - 1);
+                    pm_pending = false;
+                }
             }
             mbar_wait(&bars.g_done, b & 1, &dead, a.status);
             tc_fence_after_sync();
@@ -540,10 +565,12 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             } else {
                 mbar_arrive(&bars.a_ready);
             }
+            if (pm_pending) pm_rows(b - 1);
         };
         g_epilogue(0);
         for (int b = 0; b < nblk; ++b) {
             if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
+            else if (x >= kC) pm_rows(b);
             const float *sc = gb + (b & 3) * kGbFloats;
             mbar_wait(&bars.d1_done, b & 1, &dead, a.status);
             mbar_wait(&bars.up_done, b & 1, &dead, a.status);
@@ -585,7 +612,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&bars.o_done[b & 1]);
+            mbar_arrive(&bars.o_done[b & 3]);
             mbar_arrive(&bars.o_staged);
         }
     } else {
@@ -629,9 +656,14 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 tmem_ld_wait();
                 float v[16];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < 16; c += 4) {
                     const int t = 32 * half + 16 * q + c;
-                    v[c] = sc[kC + t] * (__bfloat162float(vt[t * kD + j]) - sc[2 * kC + t] * __uint_as_float(rr[c]));
+                    const float4 be = *reinterpret_cast<const float4 *>(sc + kC + t);
+                    const float4 ga = *reinterpret_cast<const float4 *>(sc + 2 * kC + t);
+                    v[c] = be.x * (__bfloat162float(vt[t * kD + j]) - ga.x * __uint_as_float(rr[c]));
+                    v[c + 1] = be.y * (__bfloat162float(vt[(t + 1) * kD + j]) - ga.y * __uint_as_float(rr[c + 1]));
+                    v[c + 2] = be.z * (__bfloat162float(vt[(t + 2) * kD + j]) - ga.z * __uint_as_float(rr[c + 2]));
+                    v[c + 3] = be.w * (__bfloat162float(vt[(t + 3) * kD + j]) - ga.w * __uint_as_float(rr[c + 3]));
                 }
                 store_row_chunks(sm + kOffR, j, 4 * half + 2 * q, v);
             }
@@ -649,7 +681,13 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 tmem_ld_wait();
                 float v[16];
 #pragma unroll
-                for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]) * sc[3 * kC + 32 * half + 16 * q + c];
+                for (int c = 0; c < 16; c += 4) {
+                    const float4 w4 = *reinterpret_cast<const float4 *>(sc + 3 * kC + 32 * half + 16 * q + c);
+                    v[c] = __uint_as_float(rr[c]) * w4.x;
+                    v[c + 1] = __uint_as_float(rr[c + 1]) * w4.y;
+                    v[c + 2] = __uint_as_float(rr[c + 2]) * w4.z;
+                    v[c + 3] = __uint_as_float(rr[c + 3]) * w4.w;
+                }
                 store_row_chunks(sm + kOffUw, j, 4 * half + 2 * q, v);
             }
             fence_async_smem();
@@ -692,7 +730,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 tc_fence_before_sync();
                 mbar_arrive(&bars.st_ready);
             }
-            mbar_arrive(&bars.chain_done[b & 1]);
+            mbar_arrive(&bars.chain_done[b & 3]);
         }
     }
     tc_fence_before_sync();

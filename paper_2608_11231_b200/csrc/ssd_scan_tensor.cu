@@ -122,6 +122,14 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 const int st = b & 1;
                 unsigned char *base = sm + st * kStageBytes;
                 const int row = t_begin + b * kQ;
+                // the two-stage ring cannot hide the DRAM latency of the tile loads: pull the tiles of block b+2 into L2 now
+                if (b + 2 < nblk) {
+                    tma_prefetch_l2_2d(&mapX, h * kP, row + 2 * kQ);
+                    for (int kb = 0; kb < 2; ++kb) {
+                        tma_prefetch_l2_2d(&mapB, grp * kN + kb * 64, row + 2 * kQ);
+                        tma_prefetch_l2_2d(&mapC, grp * kN + kb * 64, row + 2 * kQ);
+                    }
+                }
                 if (b < nblk) {
                     // B and C of block b-2 are free after its (d)
                     if (b >= 2) mbar_wait(&bars.bc_free[st], ((b - 2) >> 1) & 1, &dead, a.status);
