@@ -7,6 +7,7 @@ recompute segment from the composed state (both families when the workload has b
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg2|cfg3|cfg4] [--impl reference]
     python bench.py --sweep        # microseconds per exact composition against K (a JSON line of its own)
+    python bench.py --artifacts    # time of building the cached chunk states / transitions (a JSON line of its own)
 
 Prints ONE JSON line (rank 0).  `value` = context tokens served per second by the step (all requests'
 context tokens / step time), device-timed with inputs resident in HBM; `e2e` = the same with every
@@ -506,6 +507,62 @@ def run_sweep(args):
                           "about 2 us of launch gap), L2 flushed before each, median", rows=rows)))
 
 
+def run_artifacts(args):
+    """--artifacts: time of building the cached artefacts of a batch of cache chunks (64 chunks x 1024 tokens per
+    family, benchmark shapes): final-state-only scans from the empty state for S_local, and the chunk transitions /
+    log-decays.  Prints one JSON line of its own."""
+    import torch
+
+    from paper_2608_11231_b200 import binding as b
+    torch.cuda.set_device(0)
+    b.load()
+    n_chunks, L = 64, 1024
+    T = n_chunks * L
+    cu = (np.arange(n_chunks + 1) * L).astype(np.int32)
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    bf = torch.bfloat16
+    rn = lambda *shape: torch.randn(shape, generator=gen, device="cuda")
+    s, m = GDN_SHAPE, SSD_SHAPE
+    k = torch.nn.functional.normalize(rn(T, s["H_k"], s["d_k"]), dim=-1).to(bf)
+    q = torch.nn.functional.normalize(rn(T, s["H_k"], s["d_k"]), dim=-1).to(bf)
+    v = rn(T, s["H_v"], s["d_v"]).to(bf)
+    g = -0.1 * torch.nn.functional.softplus(rn(T, s["H_v"]))
+    beta = torch.sigmoid(rn(T, s["H_v"]))
+    x = rn(T, m["H"], m["P"]).to(bf)
+    dt = torch.nn.functional.softplus(-2.0 + 0.5 * rn(T, m["H"]))
+    A = -torch.exp(2.0 * torch.rand(m["H"], generator=gen, device="cuda"))
+    Bm = (rn(T, m["G"], m["N"]) / m["N"] ** 0.5).to(bf)
+    Cm = (rn(T, m["G"], m["N"]) / m["N"] ** 0.5).to(bf)
+    ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    st_g = torch.empty((n_chunks, s["H_v"], s["d_k"], s["d_v"]), device="cuda")
+    tr_g = torch.empty((n_chunks, s["H_v"], s["d_k"], s["d_k"]), device="cuda")
+    st_m = torch.empty((n_chunks, m["H"], m["N"], m["P"]), device="cuda")
+    lam = torch.empty((n_chunks, m["H"]), device="cuda")
+    calls = {
+        "gdn_states": lambda: b.lkv_gdn_fwd(q, k, v, g, beta, None, None, st_g, cu_seqlens=cu, want_outputs=False, workspace_t=ws),
+        "gdn_transitions": lambda: b.lkv_gdn_chunk_transition(k, g, beta, tr_g, cu_seqlens=cu, workspace_t=ws),
+        "mamba_states": lambda: b.lkv_ssd_fwd(x, dt, A, Bm, Cm, None, None, st_m, cu_seqlens=cu, want_outputs=False, workspace_t=ws),
+        "mamba_logdecays": lambda: b.lkv_mamba_chunk_logdecay(dt, A, lam, cu_seqlens=cu, workspace_t=ws),
+    }
+    out = {}
+    for name, fn in calls.items():
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(args.steps, 5)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        us = statistics.median(ts)
+        out[name] = dict(us=round(us, 1), tokens_per_s=round(T / us * 1e6))
+    print(json.dumps(dict(artifacts="chunk_prefill", chunks=n_chunks, chunk_len=L, timing="CUDA events around one call, "
+                          "inputs (about 1.1 GB per family) larger than L2, median", calls=out)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -514,8 +571,11 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="composition time against K instead of the step benchmark")
+    ap.add_argument("--artifacts", action="store_true", help="time of building chunk states and transitions")
     args = ap.parse_args()
-    if args.sweep:
+    if args.artifacts:
+        run_artifacts(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)

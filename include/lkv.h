@@ -242,7 +242,8 @@ int lkv_init_state_batched_static(const void *states, const void *transitions, c
  * evaluated chunkwise: inside a block of tokens the triangular system that
  * couples the tokens (WY / UT transform) is solved at once, and the state is
  * carried from block to block.  S0 == NULL starts from the empty state;
- * S_T == NULL skips the final-state write; S_T may alias S0.  Sequences of
+ * S_T == NULL skips the final-state write; S_T may alias S0; o == NULL skips
+ * the outputs (final states only; S_T is then required).  Sequences of
  * any length >= 0 are accepted (no padding is required).
  */
 int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
@@ -257,6 +258,29 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
  */
 int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
                 const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream);
+
+/*
+ * Producers of the cached artefacts that exact composition consumes (Eq. 5: a chunk C maps an incoming
+ * state as S_out = T_C S_in + S_local).  S_local of a chunk is the final state of a scan of the chunk from
+ * the empty state: call lkv_gdn_fwd / lkv_ssd_fwd with S0 == NULL and the chunks as sequences (o / y may
+ * be NULL there when only final states are wanted).  The two calls below give the other half, T_C.
+ *
+ * lkv_gdn_chunk_transition: for every sequence (= cache chunk) c of `cu_seqlens` and every value head h,
+ *     T_c = prod_t exp(g_t) (I - beta_t k_t k_t^T)      (Eq. 3; later tokens on the left)
+ * written to transitions[c][h] as a row-major d_k x d_k fp32 matrix (device, n_seq x H_v x d_k x d_k), the
+ * layout lkv_init_state reads.  It is the scan run from S = I with v = 0, so `d` is the descriptor of
+ * lkv_gdn_fwd on the same tokens (d_v must equal d_k; scale is ignored); k, g, beta as in lkv_gdn_fwd.
+ * An empty chunk gives the identity.  Precision is that of the scan path `d->compute` selects.
+ *
+ * lkv_mamba_chunk_logdecay: for every sequence c and head h, lambda[c][h] = A_h * sum_t dt_t (fp32, device,
+ * n_seq x H): exp(lambda) is the scalar T_c of Eq. 2 / Eq. 5, kept as a logarithm because it underflows
+ * fp32 for long chunks.  `d` is the descriptor of lkv_ssd_fwd on the same tokens (P, N, G unused).
+ *
+ * Errors as for the scans (LKV_ERR_DIM if d_v != d_k).  Both need the scan workspace.
+ */
+int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, float *transitions,
+                             const lkv_gdn_desc *d, void *stream);
+int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream);
 
 /*
  * Workspace size in bytes for a call described by `desc` (lkv_init_desc, lkv_gdn_desc or

@@ -28,7 +28,7 @@ LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
 LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
-           "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
+           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
 
 
 class lkv_init_desc(ctypes.Structure):
@@ -76,6 +76,8 @@ def load() -> ctypes.CDLL:
         lib.lkv_init_state_batched_static.restype = ci
         lib.lkv_gdn_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), vp]
         lib.lkv_ssd_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_ssd_desc), vp]
+        lib.lkv_gdn_chunk_transition.argtypes = [vp] * 4 + [ctypes.POINTER(lkv_gdn_desc), vp]
+        lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_workspace_bytes.argtypes = [ci, vp, ci, ci]
         lib.lkv_workspace_bytes.restype = ctypes.c_size_t
         lib.lkv_device_status.argtypes = [vp, vp]
@@ -219,11 +221,11 @@ def lkv_init_state_batched_static(states: torch.Tensor, transitions: Optional[to
 
 
 def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None, scale: float = 0.0,
-                compute: int = LKV_COMPUTE_AUTO, want_final_state: bool = True,
+                compute: int = LKV_COMPUTE_AUTO, want_final_state: bool = True, want_outputs: bool = True,
                 workspace_t: Optional[torch.Tensor] = None, stream=None):
     """Gated DeltaNet scan.  q, k: [T, H_k, d_k]; v: [T, H_v, d_v]; g, beta: [T, H_v] fp32.
 
-    Returns (o [T, H_v, d_v] in the dtype of v, S_T [n_seq, H_v, d_k, d_v] fp32 or None).
+    Returns (o [T, H_v, d_v] in the dtype of v, or None with want_outputs=False; S_T [n_seq, H_v, d_k, d_v] fp32 or None).
     """
     T, H_k, d_k = q.shape
     _, H_v, d_v = v.shape
@@ -234,7 +236,7 @@ def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None,
                      workspace=None, workspace_bytes=0)
     ws_t = workspace_t if workspace_t is not None else workspace(v.device, lkv_workspace_bytes(LKV_WS_GDN, d, n_seq))
     d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
-    if o is None:
+    if o is None and want_outputs:
         o = torch.empty_like(v)
     if S_T is None and want_final_state:
         S_T = torch.empty((n_seq, H_v, d_k, d_v), dtype=torch.float32, device=v.device)
@@ -246,7 +248,8 @@ def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None,
 
 
 def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, compute: int = LKV_COMPUTE_AUTO,
-                want_final_state: bool = True, workspace_t: Optional[torch.Tensor] = None, stream=None):
+                want_final_state: bool = True, want_outputs: bool = True,
+                workspace_t: Optional[torch.Tensor] = None, stream=None):
     """Mamba-2 (SSD) scan.  x: [T, H, P]; dt: [T, H] fp32; A: [H] fp32; B, C: [T, G, N].
 
     Returns (y [T, H, P] in the dtype of x, S_T [n_seq, H, N, P] fp32 or None).
@@ -259,7 +262,7 @@ def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, c
                      io_dtype=_dtype_code(x), compute=compute, workspace=None, workspace_bytes=0)
     ws_t = workspace_t if workspace_t is not None else workspace(x.device, lkv_workspace_bytes(LKV_WS_SSD, d, n_seq))
     d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
-    if y is None:
+    if y is None and want_outputs:
         y = torch.empty_like(x)
     if S_T is None and want_final_state:
         S_T = torch.empty((n_seq, H, N, P), dtype=torch.float32, device=x.device)
@@ -268,3 +271,44 @@ def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, c
     if st != LKV_OK:
         raise LkvError(st, "lkv_ssd_fwd")
     return y, S_T
+
+
+def lkv_gdn_chunk_transition(k, g, beta, transitions=None, *, cu_seqlens=None, H_v: Optional[int] = None,
+                             compute: int = LKV_COMPUTE_AUTO, workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """Accumulated transition of every chunk (sequence of cu_seqlens) and value head.
+
+    k: [T, H_k, d]; g, beta: [T, H_v] fp32.  Returns transitions [n_seq, H_v, d, d] fp32.
+    """
+    T, H_k, d_k = k.shape
+    H_v = g.shape[1] if H_v is None else H_v
+    cu = _host_i32(cu_seqlens)
+    n_seq = 1 if cu is None else cu.size - 1
+    d = lkv_gdn_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H_k=H_k, H_v=H_v,
+                     d_k=d_k, d_v=d_k, io_dtype=_dtype_code(k), compute=compute, scale=0.0, reserved=0,
+                     workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(k.device, lkv_workspace_bytes(LKV_WS_GDN, d, n_seq))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    if transitions is None:
+        transitions = torch.empty((n_seq, H_v, d_k, d_k), dtype=torch.float32, device=k.device)
+    st = load().lkv_gdn_chunk_transition(_ptr(k), _ptr(g), _ptr(beta), _ptr(transitions), ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_gdn_chunk_transition")
+    return transitions
+
+
+def lkv_mamba_chunk_logdecay(dt, A, logdecay=None, *, cu_seqlens=None, workspace_t: Optional[torch.Tensor] = None,
+                             stream=None):
+    """lambda[c][h] = A[h] * sum of dt over chunk c.  dt: [T, H] fp32; A: [H] fp32.  Returns [n_seq, H] fp32."""
+    T, H = dt.shape
+    cu = _host_i32(cu_seqlens)
+    n_seq = 1 if cu is None else cu.size - 1
+    d = lkv_ssd_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H=H, P=1, N=1, G=1,
+                     io_dtype=LKV_DTYPE_F32, compute=LKV_COMPUTE_AUTO, workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(dt.device, lkv_workspace_bytes(LKV_WS_SSD, d, n_seq))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    if logdecay is None:
+        logdecay = torch.empty((n_seq, H), dtype=torch.float32, device=dt.device)
+    st = load().lkv_mamba_chunk_logdecay(_ptr(dt), _ptr(A), _ptr(logdecay), ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_mamba_chunk_logdecay")
+    return logdecay

@@ -65,6 +65,8 @@ struct GdnArgs {
     float *S_T;
     int32_t n_seq, T_total, H_k, H_v, d_k, d_v;
     float scale;
+    int32_t s0_identity;         // start every sequence from S = I (d_k == d_v) instead of S0; with v == nullptr (read
+                                 // as zeros) the final state is then the sequence's accumulated transition; o may be nullptr
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
 };
@@ -95,5 +97,7 @@ bool ssd_scan_fp32_supported(int N, int P);
 cudaError_t launch_ssd_scan_fp32(const SsdArgs &a, bool io_bf16, cudaStream_t s);
 bool ssd_scan_tensor_supported(const SsdArgs &a, bool io_bf16);
 cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s);
+// lambda[c][h] = A[h] * sum of dt over sequence c (cu in the parameter block of `a`; only dt, A, H, n_seq, cu are read)
+cudaError_t launch_mamba_logdecay(const SsdArgs &a, float *logdecay, cudaStream_t s);
 
 }  // namespace lkv

@@ -48,7 +48,8 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
     T *o = static_cast<T *>(a.o);
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * dk * DV;
 
-    for (int idx = tid; idx < dk * DV; idx += 256) S[idx] = a.S0 ? a.S0[sbase + idx] : 0.f;
+    for (int idx = tid; idx < dk * DV; idx += 256)
+        S[idx] = a.s0_identity ? (idx / DV == idx % DV ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + idx] : 0.f);
 
     for (int t0 = t_begin; t0 < t_end; t0 += kC) {
         const int n = min(kC, t_end - t0);
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
         }
         for (int idx = tid; idx < kC * DV; idx += 256) {
             const int t = idx / DV, c = idx % DV;
-            Vs[idx] = t < n ? to_f32<T>(v[(static_cast<size_t>(t0 + t) * a.H_v + h) * DV + c]) : 0.f;
+            Vs[idx] = (v && t < n) ? to_f32<T>(v[(static_cast<size_t>(t0 + t) * a.H_v + h) * DV + c]) : 0.f;
         }
         if (tid < kC) {
             const bool ok = tid < n;  // a padded token is the identity step: g = 0, beta = 0
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
             const int t = tg + NG * u;
             float acc = expf(cg[t]) * qS[u];
             for (int i = 0; i <= t; ++i) acc = fmaf(Pm[t * (kC + 1) + i], Us[i * DV + j], acc);
-            if (t < n) o[(static_cast<size_t>(t0 + t) * a.H_v + h) * DV + j] = from_f32<T>(a.scale * acc);
+            if (o && t < n) o[(static_cast<size_t>(t0 + t) * a.H_v + h) * DV + j] = from_f32<T>(a.scale * acc);
         }
         // state carry: thread (tg, j) owns rows tg, tg + NG, ... of column j
         {

@@ -196,8 +196,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * kD * kD;
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
-        if (a.S_T && a.S_T != a.S0)
-            for (int e = tid; e < kD * kD; e += kThreads) a.S_T[sbase + e] = a.S0 ? a.S0[sbase + e] : 0.f;
+        if (a.S_T && (a.S_T != a.S0 || a.s0_identity))
+            for (int e = tid; e < kD * kD; e += kThreads)
+                a.S_T[sbase + e] = a.s0_identity ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f);
         return;
     }
     if (tid == 0) {
@@ -224,7 +225,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         if (lane == 0) {
             tma_prefetch_desc(&mapQ);
             tma_prefetch_desc(&mapK);
-            tma_prefetch_desc(&mapV);
+            if (a.v) tma_prefetch_desc(&mapV);
             for (int b = 0; b < nblk; ++b) {
                 const int st = b & 1;
                 const int row = t_begin + b * kC;
@@ -234,7 +235,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                         tma_prefetch_l2_2d(&mapQ, hk * kD + kb * 64, row + 2 * kC);
                         tma_prefetch_l2_2d(&mapK, hk * kD + kb * 64, row + 2 * kC);
                     }
-                    tma_prefetch_l2_2d(&mapV, h * kD, row + 2 * kC);
+                    if (a.v) tma_prefetch_l2_2d(&mapV, h * kD, row + 2 * kC);
                 }
                 if (b >= 2) mbar_wait(&bars.tiles_free_qk[st], ((b - 2) >> 1) & 1, &dead, a.status);
                 unsigned char *base = sm + st * kQKStage;
@@ -243,9 +244,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     tma_load_2d(base + kb * 2 * kC * 128, &mapQ, hk * kD + kb * 64, row, &bars.full_qk[st]);
                     tma_load_2d(base + kb * 2 * kC * 128 + kC * 128, &mapK, hk * kD + kb * 64, row, &bars.full_qk[st]);
                 }
-                if (b >= 1) mbar_wait(&bars.v_free, (b - 1) & 1, &dead, a.status);
-                mbar_expect_tx(&bars.full_v, kC * kD * 2);
-                tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
+                if (a.v) {   // without v (read as zeros) nothing is loaded and the chain does not wait for it
+                    if (b >= 1) mbar_wait(&bars.v_free, (b - 1) & 1, &dead, a.status);
+                    mbar_expect_tx(&bars.full_v, kC * kD * 2);
+                    tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
+                }
             }
         }
     } else if (warp == 19) {
@@ -300,11 +303,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     } else if (warp == 18) {
         // ======================================================= TMA store of the output tiles (whole blocks only)
         if (lane == 0) {
-            tma_prefetch_desc(&mapO);
+            if (a.o) tma_prefetch_desc(&mapO);
             for (int b = 0; b < nblk; ++b) {
                 mbar_wait(&bars.o_staged, b & 1, &dead, a.status);
                 const int t0 = t_begin + b * kC;
-                if (t0 + kC <= t_end && !dead) {
+                if (a.o && t0 + kC <= t_end && !dead) {
                     tma_store_2d(&mapO, sm + kOffMPM + (b & 1) * (kD * 128), h * kD, t0);
                     tma_store_commit();
                     tma_store_wait_read();
@@ -577,7 +580,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tc_fence_after_sync();
             const int t0 = t_begin + b * kC;
             const int n = min(kC, t_end - t0);
-            if (n == kC) {
+            if (!a.o) {
+                // no outputs wanted (final state only): nothing to drain
+            } else if (n == kC) {
                 // whole block: stage the tile [token][j] in the [M; PM] buffer of this block, which (3) has finished
                 // reading (up_done); the store warp writes it out with TMA
                 __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffMPM + (b & 1) * (kD * 128)) + j;
@@ -629,7 +634,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 uint32_t rr[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    v[c] = a.S0 ? a.S0[sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j] : 0.f;
+                    const int m = 64 * half + 16 * q + c;
+                    v[c] = a.s0_identity ? (m == j ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + static_cast<size_t>(m) * kD + j] : 0.f);
                     rr[c] = __float_as_uint(v[c] * gamC);
                 }
                 tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);
@@ -645,7 +651,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const float *sc = gb + (b & 3) * kGbFloats;
             const __nv_bfloat16 *vt = reinterpret_cast<const __nv_bfloat16 *>(sm + kOffV);
             if (b > 0) mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
-            mbar_wait(&bars.full_v, par, &dead, a.status);
+            const bool has_v = a.v != nullptr;
+            if (has_v) mbar_wait(&bars.full_v, par, &dead, a.status);
             mbar_wait(&bars.d1_done, par, &dead, a.status);
             tc_fence_after_sync();
             // r_t = beta_t (v_t[j] - gam_t (S^T k_t)_j), t = 32*half..+31 -> R^T row j
@@ -660,10 +667,14 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     const int t = 32 * half + 16 * q + c;
                     const float4 be = *reinterpret_cast<const float4 *>(sc + kC + t);
                     const float4 ga = *reinterpret_cast<const float4 *>(sc + 2 * kC + t);
-                    v[c] = be.x * (__bfloat162float(vt[t * kD + j]) - ga.x * __uint_as_float(rr[c]));
-                    v[c + 1] = be.y * (__bfloat162float(vt[(t + 1) * kD + j]) - ga.y * __uint_as_float(rr[c + 1]));
-                    v[c + 2] = be.z * (__bfloat162float(vt[(t + 2) * kD + j]) - ga.z * __uint_as_float(rr[c + 2]));
-                    v[c + 3] = be.w * (__bfloat162float(vt[(t + 3) * kD + j]) - ga.w * __uint_as_float(rr[c + 3]));
+                    const float v0 = has_v ? __bfloat162float(vt[t * kD + j]) : 0.f;
+                    const float v1 = has_v ? __bfloat162float(vt[(t + 1) * kD + j]) : 0.f;
+                    const float v2 = has_v ? __bfloat162float(vt[(t + 2) * kD + j]) : 0.f;
+                    const float v3 = has_v ? __bfloat162float(vt[(t + 3) * kD + j]) : 0.f;
+                    v[c] = be.x * (v0 - ga.x * __uint_as_float(rr[c]));
+                    v[c + 1] = be.y * (v1 - ga.y * __uint_as_float(rr[c + 1]));
+                    v[c + 2] = be.z * (v2 - ga.z * __uint_as_float(rr[c + 2]));
+                    v[c + 3] = be.w * (v3 - ga.w * __uint_as_float(rr[c + 3]));
                 }
                 store_row_chunks(sm + kOffR, j, 4 * half + 2 * q, v);
             }
@@ -750,9 +761,11 @@ cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s) {
     const uint64_t qk_inner = static_cast<uint64_t>(a.H_k) * kD, v_inner = static_cast<uint64_t>(a.H_v) * kD;
     if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         !make_tensor_map_2d(&mapK, a.k, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
-        !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, kD, kC, false) ||
-        !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false))
+        (a.v && !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, kD, kC, false)) ||
+        (a.o && !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false)))
         return cudaErrorInvalidValue;
+    if (!a.v) mapV = mapK;   // never used by the kernel then
+    if (!a.o) mapO = mapK;
     // dynamic shared memory: everything the device allows beside the kernel's static part (the map needs
     // kSmemUsed bytes from a 1024-byte aligned base; the kernel checks that it fits)
     cudaFuncAttributes fa;

@@ -206,4 +206,33 @@ cudaError_t launch_init_gdn_exact_fp32(const InitArgs &a, bool pool_bf16, cudaSt
     return cudaGetLastError();
 }
 
+namespace {
+
+// One warp per (sequence, group of 32 heads): lanes walk consecutive heads, so every token's dt row is read with
+// coalesced 128-byte accesses; four partial sums per lane keep several loads in flight.
+__global__ void mamba_logdecay_kernel(const __grid_constant__ SsdArgs a, float *__restrict__ out) {
+    const int seq = blockIdx.y;
+    const int h = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int part = threadIdx.x >> 5, nparts = blockDim.x >> 5;
+    __shared__ float red[8][32];
+    const int t0 = a.cu[seq], t1 = a.cu[seq + 1];
+    float acc = 0.f;
+    if (h < a.H)
+        for (int t = t0 + part; t < t1; t += nparts) acc += a.dt[static_cast<size_t>(t) * a.H + h];
+    red[part][threadIdx.x & 31] = acc;
+    __syncthreads();
+    if (part == 0 && h < a.H) {
+        float sum = 0.f;
+        for (int p = 0; p < nparts; ++p) sum += red[p][threadIdx.x];
+        out[static_cast<size_t>(seq) * a.H + h] = a.A[h] * sum;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_mamba_logdecay(const SsdArgs &a, float *logdecay, cudaStream_t s) {
+    mamba_logdecay_kernel<<<dim3((a.H + 31) / 32, a.n_seq), 256, 0, s>>>(a, logdecay);
+    return cudaGetLastError();
+}
+
 }  // namespace lkv

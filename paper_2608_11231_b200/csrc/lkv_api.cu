@@ -170,8 +170,9 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
     return init_impl(states, transitions, chunk_ids, cu_k, n_req, mode, sel_index, S0, d, stream);
 }
 
-int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
-                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream) {
+// lkv_gdn_fwd, and with `transition` set the scan from S = I with v = 0 whose final state is the chunk transition
+static int gdn_impl(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                    const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream, bool transition) {
     if (!d) return LKV_ERR_NULL;
     if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
     if (d->H_k < 1 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1 || d->H_v % d->H_k != 0) return LKV_ERR_DIM;
@@ -179,7 +180,10 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
     int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
     if (st != LKV_OK) return st;
     if (d->n_seq == 0) return LKV_OK;
-    if (d->T_total > 0 && (!q || !k || !v || !g || !beta || !o)) return LKV_ERR_NULL;
+    if (transition && d->d_k != d->d_v) return LKV_ERR_DIM;
+    if (d->T_total > 0 && (!q || !k || !g || !beta)) return LKV_ERR_NULL;
+    if (!transition && d->T_total > 0 && !v) return LKV_ERR_NULL;
+    if (!o && !S_T) return LKV_ERR_NULL;   // nothing to compute
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(S0) ||
         !aligned16(o) || !aligned16(S_T))
         return LKV_ERR_ALIGN;
@@ -190,6 +194,7 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
     a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = S_T;
     a.n_seq = d->n_seq; a.T_total = d->T_total; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
     a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
+    a.s0_identity = transition ? 1 : 0;
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
     const bool tensor_fits = gdn_scan_tensor_supported(a, io_bf16);
@@ -212,6 +217,38 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
     return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
 }
 
+int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream) {
+    return gdn_impl(q, k, v, g, beta, S0, o, S_T, d, stream, false);
+}
+
+int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, float *transitions,
+                             const lkv_gdn_desc *d, void *stream) {
+    if (d && d->n_seq > 0 && !transitions) return LKV_ERR_NULL;
+    // q is not needed for the state: the key tensor stands in for it (its read-outs are not written)
+    return gdn_impl(k, k, nullptr, g, beta, nullptr, nullptr, transitions, d, stream, true);
+}
+
+int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (d->H < 1) return LKV_ERR_DIM;
+    std::vector<int32_t> cu;
+    int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
+    if (st != LKV_OK) return st;
+    if (d->n_seq == 0) return LKV_OK;
+    if (!A || !logdecay || (d->T_total > 0 && !dt)) return LKV_ERR_NULL;
+    if (!aligned16(dt) || !aligned16(A) || !aligned16(logdecay)) return LKV_ERR_ALIGN;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+    SsdArgs a{};
+    a.dt = dt; a.A = A; a.n_seq = d->n_seq; a.T_total = d->T_total; a.H = d->H; a.P = d->P; a.N = d->N; a.G = d->G;
+    a.status = static_cast<int32_t *>(d->workspace);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = place_indices(a.cu, cu, d->workspace, s);
+    if (st != LKV_OK) return st;
+    return launch_mamba_logdecay(a, logdecay, s) == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
 int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
                 const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream) {
     if (!d) return LKV_ERR_NULL;
@@ -222,7 +259,8 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
     if (st != LKV_OK) return st;
     if (d->n_seq == 0) return LKV_OK;
     if (!A) return LKV_ERR_NULL;
-    if (d->T_total > 0 && (!x || !dt || !B || !C || !y)) return LKV_ERR_NULL;
+    if (d->T_total > 0 && (!x || !dt || !B || !C)) return LKV_ERR_NULL;
+    if (!y && !S_T) return LKV_ERR_NULL;   // nothing to compute
     if (!aligned16(x) || !aligned16(dt) || !aligned16(A) || !aligned16(B) || !aligned16(C) || !aligned16(S0) ||
         !aligned16(y) || !aligned16(S_T))
         return LKV_ERR_ALIGN;

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) ssd_scan_fp32_kernel(const __grid_constan
             const int t = tg + NG * u;
             float acc = expf(ls[t]) * cS[u];
             for (int i = 0; i <= t; ++i) acc = fmaf(Gm[t * (kQ + 1) + i], Xs[i * P + p], acc);
-            if (t < n) y[(static_cast<size_t>(t0 + t) * a.H + h) * P + p] = from_f32<T>(acc);
+            if (y && t < n) y[(static_cast<size_t>(t0 + t) * a.H + h) * P + p] = from_f32<T>(acc);
         }
         {
             float w[kQ];

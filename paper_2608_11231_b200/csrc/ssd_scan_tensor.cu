@@ -117,7 +117,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             tma_prefetch_desc(&mapX);
             tma_prefetch_desc(&mapB);
             tma_prefetch_desc(&mapC);
-            tma_prefetch_desc(&mapY);
+            if (a.y) tma_prefetch_desc(&mapY);
             for (int b = 0; b < nblk + 2; ++b) {
                 const int st = b & 1;
                 unsigned char *base = sm + st * kStageBytes;
@@ -142,7 +142,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 if (b >= 2) {
                     // the X tile of block b-2 now stages its y tile (whole blocks only): store it, then reuse the tile
                     mbar_wait(&bars.ys_ready[st], ((b - 2) >> 1) & 1, &dead, a.status);
-                    if (row - kQ <= t_end && !dead) {
+                    if (a.y && row - kQ <= t_end && !dead) {
                         tma_store_2d(&mapY, base, h * kP, row - 2 * kQ);
                         tma_store_commit();
                         tma_store_wait_read();
@@ -422,7 +422,9 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 for (int c = 0; c < 32; c += 2)
                     w[c / 2] = pack_bf16(__uint_as_float(ya[c]) + et * __uint_as_float(ye[c]),
                                          __uint_as_float(ya[c + 1]) + et * __uint_as_float(ye[c + 1]));
-                if (row0 + kQ <= t_end) {
+                if (!a.y) {
+                    // no outputs wanted (final states only)
+                } else if (row0 + kQ <= t_end) {
                     // whole block inside the sequence: stage the y tile in this block's X tile ((b) has read it) in
                     // the layout of the tensor map and let the TMA warp store it -- full 128-byte rows
                     // instead of 32 scattered 16-byte pieces per warp instruction
@@ -464,8 +466,9 @@ cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s) {
     if (!make_tensor_map_2d(&mapX, a.x, 2, x_inner, rows, x_inner * 2, 64, kQ, true) ||
         !make_tensor_map_2d(&mapB, a.B, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
         !make_tensor_map_2d(&mapC, a.C, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
-        !make_tensor_map_2d(&mapY, a.y, 2, x_inner, rows, x_inner * 2, 64, kQ, true))
+        (a.y && !make_tensor_map_2d(&mapY, a.y, 2, x_inner, rows, x_inner * 2, 64, kQ, true)))
         return cudaErrorInvalidValue;
+    if (!a.y) mapY = mapX;   // never used by the kernel then
     cudaError_t e = cudaFuncSetAttribute(ssd_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     ssd_scan_tensor_kernel<<<dim3(a.H, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapX, mapB, mapC, mapY);

@@ -142,6 +142,30 @@ def test_ssd_fwd_argument_errors(lib):
     assert f(_ssd_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE
 
 
+def test_artifact_producers_argument_errors(lib):
+    t = lambda d, k=FAKE, out=FAKE: lib.lkv_gdn_chunk_transition(k, FAKE, FAKE, out,
+                                                                  ctypes.byref(d) if d is not None else None, None)
+    assert t(None) == b.LKV_ERR_NULL
+    assert t(_gdn_desc(d_k=128, d_v=64)) == b.LKV_ERR_DIM             # the transition is d_k x d_k: d_v must equal d_k
+    assert t(_gdn_desc(), out=None) == b.LKV_ERR_NULL
+    assert t(_gdn_desc(), k=None) == b.LKV_ERR_NULL
+    assert t(_gdn_desc(), out=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert t(_gdn_desc(workspace=None)) == b.LKV_ERR_WORKSPACE
+    m = lambda d, dt=FAKE, A=FAKE, out=FAKE: lib.lkv_mamba_chunk_logdecay(dt, A, out,
+                                                                          ctypes.byref(d) if d is not None else None, None)
+    assert m(None) == b.LKV_ERR_NULL
+    assert m(_ssd_desc(H=0)) == b.LKV_ERR_DIM
+    assert m(_ssd_desc(), A=None) == b.LKV_ERR_NULL
+    assert m(_ssd_desc(), out=None) == b.LKV_ERR_NULL
+    assert m(_ssd_desc(), dt=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert m(_ssd_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE
+    # final-state-only scans: o / y may be NULL, but not together with S_T
+    g = lib.lkv_gdn_fwd(FAKE, FAKE, FAKE, FAKE, FAKE, None, None, None, ctypes.byref(_gdn_desc()), None)
+    assert g == b.LKV_ERR_NULL
+    y = lib.lkv_ssd_fwd(FAKE, FAKE, FAKE, FAKE, FAKE, None, None, None, ctypes.byref(_ssd_desc()), None)
+    assert y == b.LKV_ERR_NULL
+
+
 def test_workspace_bytes(lib):
     d = _desc()
     small = b.lkv_workspace_bytes(b.LKV_WS_INIT, d, 1, 8)

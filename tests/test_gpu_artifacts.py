@@ -1,0 +1,116 @@
+"""Producers of the cached artefacts (chunk transitions, log-decays, final-state-only scans) against the oracle,
+and the whole cache-building pipeline on the GPU: chunk tokens -> (S_local, T_C) -> exact composition, which must
+equal one sequential pass of the oracle over the concatenated prefix (Eq. 5, Eq. 6)."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import TOL_BF16, TOL_F32, dev, host, maxrel
+from paper_2608_11231_b200 import binding as b
+from paper_2608_11231_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _t():
+    import torch
+    return torch
+
+
+def _cat(chunks, names):
+    return {n: np.concatenate([c[n] for c in chunks]) for n in names}
+
+
+@pytest.mark.parametrize("shape", [
+    dict(H_k=2, H_v=4, d=64, io="f32", lens=[70, 0, 33, 128], tol=TOL_F32),
+    dict(H_k=2, H_v=4, d=128, io="bf16", lens=[200, 64, 0, 131], tol=TOL_BF16),
+    dict(H_k=1, H_v=2, d=128, io="bf16", lens=[1024], tol=TOL_BF16),
+])
+@pytest.mark.parametrize("live", [False, True])
+def test_gdn_chunk_transition_matches_oracle(shape, live):
+    torch = _t()
+    H_k, H_v, d, io = shape["H_k"], shape["H_v"], shape["d"], shape["io"]
+    rng = np.random.default_rng(11)
+    chunks = [wl.gdn_tokens(rng, L, H_k, H_v, d, d, io=io, live_chunk_len=256 if live else None) for L in shape["lens"]]
+    cat = _cat(chunks, ("k", "g", "beta"))
+    cu = np.concatenate([[0], np.cumsum(shape["lens"])]).astype(np.int32)
+    dt = torch.bfloat16 if io == "bf16" else None
+    T = host(b.lkv_gdn_chunk_transition(dev(cat["k"], dt), dev(cat["g"]), dev(cat["beta"]), cu_seqlens=cu))
+    assert T.shape == (len(chunks), H_v, d, d)
+    for c, ch in enumerate(chunks):
+        if len(ch["k"]) == 0:
+            assert T[c].tobytes() == np.broadcast_to(np.eye(d, dtype=np.float32), (H_v, d, d)).tobytes()
+            continue
+        ref = oracle.gdn_transition(ch["k"], ch["g"], ch["beta"])
+        assert maxrel(T[c], ref) <= shape["tol"], (c, maxrel(T[c], ref))
+
+
+def test_mamba_chunk_logdecay_matches_oracle():
+    rng = np.random.default_rng(12)
+    H, lens = 80, [1024, 0, 77, 300]
+    A = wl.ssd_A(rng, H)
+    dts = [wl.ssd_tokens(rng, L, H, 8, 16, 1, io="f32")["dt"] for L in lens]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    lam = host(b.lkv_mamba_chunk_logdecay(dev(np.concatenate(dts)), dev(A), cu_seqlens=cu))
+    assert lam.shape == (len(lens), H)
+    for c, d in enumerate(dts):
+        ref = oracle.mamba_logdecay(d, A) if len(d) else np.zeros(H)
+        assert np.abs(lam[c] - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max())
+
+
+def test_final_state_only_scans_equal_full_scans():
+    torch = _t()
+    bf = torch.bfloat16
+    rng = np.random.default_rng(13)
+    lens = [300, 64, 129]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    g = wl.gdn_tokens(rng, sum(lens), 2, 4, 128, 128)
+    args = (dev(g["q"], bf), dev(g["k"], bf), dev(g["v"], bf), dev(g["g"]), dev(g["beta"]))
+    o, ST = b.lkv_gdn_fwd(*args, cu_seqlens=cu)
+    o2, ST2 = b.lkv_gdn_fwd(*args, cu_seqlens=cu, want_outputs=False)
+    assert o2 is None and host(ST2).tobytes() == host(ST).tobytes()
+    m = wl.ssd_tokens(rng, sum(lens), 8, 64, 128, 1)
+    A = wl.ssd_A(rng, 8)
+    margs = (dev(m["x"], bf), dev(m["dt"]), dev(A), dev(m["B"], bf), dev(m["C"], bf))
+    y, MT = b.lkv_ssd_fwd(*margs, cu_seqlens=cu)
+    y2, MT2 = b.lkv_ssd_fwd(*margs, cu_seqlens=cu, want_outputs=False)
+    assert y2 is None and host(MT2).tobytes() == host(MT).tobytes()
+
+
+def test_cache_building_pipeline_gdn_reproduces_the_full_prefix_state():
+    """Artefacts made by the library from raw chunk tokens, composed by the library, against one oracle pass."""
+    torch = _t()
+    bf = torch.bfloat16
+    H_k, H_v, d, lens = 2, 4, 128, [256, 192, 320, 256]
+    rng = np.random.default_rng(14)
+    chunks = [wl.gdn_tokens(rng, L, H_k, H_v, d, d, live_chunk_len=256) for L in lens]
+    cat = _cat(chunks, ("q", "k", "v", "g", "beta"))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q, k, v, g, beta = dev(cat["q"], bf), dev(cat["k"], bf), dev(cat["v"], bf), dev(cat["g"]), dev(cat["beta"])
+    _, states = b.lkv_gdn_fwd(q, k, v, g, beta, cu_seqlens=cu, want_outputs=False)      # S_local of every chunk
+    trans = b.lkv_gdn_chunk_transition(k, g, beta, cu_seqlens=cu)                        # T_C of every chunk
+    S0 = host(b.lkv_init_state(states, trans, len(lens), b.LKV_INIT_EXACT, family=b.LKV_FAMILY_GDN))
+    _, S_ref = oracle.gdn_seq(cat["q"], cat["k"], cat["v"], cat["g"], cat["beta"])
+    assert maxrel(S0, S_ref) <= TOL_BF16, maxrel(S0, S_ref)
+    # the carried part (everything but the last chunk's own state) is what composition adds
+    last = host(states)[-1].astype(np.float64)
+    carried_ref = S_ref - oracle.gdn_seq(*[chunks[-1][n] for n in ("q", "k", "v", "g", "beta")])[1]
+    assert np.abs(carried_ref).max() > 0.05 * np.abs(S_ref).max()
+    assert maxrel(S0 - last, carried_ref) <= 2 * TOL_BF16
+
+
+def test_cache_building_pipeline_mamba_reproduces_the_full_prefix_state():
+    torch = _t()
+    bf = torch.bfloat16
+    H, P, N, lens = 8, 64, 128, [256, 128, 384]
+    rng = np.random.default_rng(15)
+    A = wl.ssd_A(rng, H, live_chunk_len=256)
+    chunks = [wl.ssd_tokens(rng, L, H, P, N, 1) for L in lens]
+    cat = _cat(chunks, ("x", "dt", "B", "C"))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    x, dt, Bm, Cm = dev(cat["x"], bf), dev(cat["dt"]), dev(cat["B"], bf), dev(cat["C"], bf)
+    _, states = b.lkv_ssd_fwd(x, dt, dev(A), Bm, Cm, cu_seqlens=cu, want_outputs=False)
+    lam = b.lkv_mamba_chunk_logdecay(dt, dev(A), cu_seqlens=cu)
+    S0 = host(b.lkv_init_state(states, lam, len(lens), b.LKV_INIT_EXACT, family=b.LKV_FAMILY_MAMBA2))
+    _, S_ref = oracle.ssd_seq(cat["x"], cat["dt"], A, cat["B"], cat["C"])
+    assert maxrel(S0, S_ref) <= TOL_BF16, maxrel(S0, S_ref)
