@@ -283,6 +283,19 @@ int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, f
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream);
 
 /*
+ * Diagnostic of Section 3.2 ("Diagnosis via relative error"): how far a constructed initial state is from the
+ * true full-prefix state, rel_err[i] = ||S_init_i - S_ref_i||_F / ||S_ref_i||_F for i < n_states, where state i
+ * is the i-th run of state_elems consecutive fp32 values of S_init / S_ref (device; a run may be one head's
+ * state, one request's, or a whole layer's).  rel_err: n_states fp32 (device).  state_elems must be a positive
+ * multiple of 4 and both arrays 16-byte aligned.  The workspace (device, 16-byte aligned) holds the partial sums:
+ * at least lkv_state_rel_error_workspace_bytes(n_states, state_elems) bytes.  Sums are fp32 accumulated in a
+ * fixed order (deterministic).  A zero reference gives inf (nan if the constructed state is zero too).
+ */
+int lkv_state_rel_error(const float *S_init, const float *S_ref, float *rel_err, int n_states, size_t state_elems,
+                        void *workspace, size_t workspace_bytes, void *stream);
+size_t lkv_state_rel_error_workspace_bytes(int n_states, size_t state_elems);
+
+/*
  * Workspace size in bytes for a call described by `desc` (lkv_init_desc, lkv_gdn_desc or
  * lkv_ssd_desc according to `which`).  n_units is the number of requests (init) or
  * sequences (scans) and n_index the total number of chunk ids over all requests

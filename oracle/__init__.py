@@ -198,3 +198,19 @@ def init_single(states, chunk_ids=None, K=None, b=None):
         b = K - 1
     assert 0 <= b < K
     return states[ids[b]].copy(), int(ids[b])
+
+
+def state_rel_error(S_init, S_ref, n_states=None):
+    """Relative error of constructed states against reference states, one number per state:
+    ||S_init_i - S_ref_i|| / ||S_ref_i|| in the Frobenius norm (Section 3.2, "Diagnosis via relative error").
+
+    The arrays are split into ``n_states`` equal parts along the flattened leading order (default: the
+    leading axis).  A zero reference gives inf, or nan when the constructed state is zero too.
+    """
+    a, r = _f64(S_init), _f64(S_ref)
+    assert a.shape == r.shape
+    n = a.shape[0] if n_states is None else int(n_states)
+    a, r = a.reshape(n, -1), r.reshape(n, -1)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        return np.sqrt(((a - r) ** 2).sum(axis=1)) / np.sqrt((r ** 2).sum(axis=1))
+

@@ -28,7 +28,8 @@ LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
 LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
-           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
+           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_state_rel_error",
+           "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
 
 
 class lkv_init_desc(ctypes.Structure):
@@ -78,6 +79,9 @@ def load() -> ctypes.CDLL:
         lib.lkv_ssd_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_gdn_chunk_transition.argtypes = [vp] * 4 + [ctypes.POINTER(lkv_gdn_desc), vp]
         lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
+        lib.lkv_state_rel_error.argtypes = [vp, vp, vp, ci, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
+        lib.lkv_state_rel_error_workspace_bytes.argtypes = [ci, ctypes.c_size_t]
+        lib.lkv_state_rel_error_workspace_bytes.restype = ctypes.c_size_t
         lib.lkv_workspace_bytes.argtypes = [ci, vp, ci, ci]
         lib.lkv_workspace_bytes.restype = ctypes.c_size_t
         lib.lkv_device_status.argtypes = [vp, vp]
@@ -312,3 +316,21 @@ def lkv_mamba_chunk_logdecay(dt, A, logdecay=None, *, cu_seqlens=None, workspace
     if st != LKV_OK:
         raise LkvError(st, "lkv_mamba_chunk_logdecay")
     return logdecay
+
+
+def lkv_state_rel_error(S_init, S_ref, n_states: Optional[int] = None, rel_err=None, *, stream=None):
+    """||S_init_i - S_ref_i|| / ||S_ref_i|| per state; the tensors are split into n_states equal runs
+    (default: along the leading axis).  Returns rel_err [n_states] fp32."""
+    assert S_init.shape == S_ref.shape and S_init.dtype == torch.float32 and S_ref.dtype == torch.float32
+    n = S_init.shape[0] if n_states is None else int(n_states)
+    elems = S_init.numel() // max(n, 1)
+    if rel_err is None:
+        rel_err = torch.empty((n,), dtype=torch.float32, device=S_init.device)
+    nbytes = load().lkv_state_rel_error_workspace_bytes(n, elems)
+    ws_t = workspace(S_init.device, max(int(nbytes), 256))
+    st = load().lkv_state_rel_error(_ptr(S_init), _ptr(S_ref), _ptr(rel_err), n, elems, ws_t.data_ptr(), ws_t.numel(),
+                                    _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_state_rel_error")
+    return rel_err
+

@@ -99,5 +99,10 @@ bool ssd_scan_tensor_supported(const SsdArgs &a, bool io_bf16);
 cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s);
 // lambda[c][h] = A[h] * sum of dt over sequence c (cu in the parameter block of `a`; only dt, A, H, n_seq, cu are read)
 cudaError_t launch_mamba_logdecay(const SsdArgs &a, float *logdecay, cudaStream_t s);
+// rel_err[i] = ||x_i - r_i|| / ||r_i|| over n_states runs of `elems` floats; parts = CTAs per state, partial sums
+// (2 floats per CTA) in `partials`
+int state_err_parts(size_t elems);
+cudaError_t launch_state_rel_error(const float *x, const float *r, float *rel_err, int n_states, size_t elems,
+                                   float *partials, cudaStream_t s);
 
 }  // namespace lkv

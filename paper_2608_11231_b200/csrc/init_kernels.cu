@@ -235,4 +235,68 @@ cudaError_t launch_mamba_logdecay(const SsdArgs &a, float *logdecay, cudaStream_
     return cudaGetLastError();
 }
 
+namespace {
+
+constexpr int kErrThreads = 256;
+constexpr size_t kErrElemsPerCta = 16384;   // 64 KB of each input per CTA: 16 float4 per thread
+
+// Squared norms of (x - r) and r over one slice of one state; one (num, den) pair per CTA, summed in a fixed order.
+__global__ void state_err_partial_kernel(const float *__restrict__ x, const float *__restrict__ r, size_t elems, int parts,
+                                         float *__restrict__ partials) {
+    const int state = blockIdx.y, part = blockIdx.x;
+    const size_t vecs = elems / 4;
+    const size_t v0 = vecs * part / parts, v1 = vecs * (part + 1) / parts;
+    const float4 *xv = reinterpret_cast<const float4 *>(x + static_cast<size_t>(state) * elems);
+    const float4 *rv = reinterpret_cast<const float4 *>(r + static_cast<size_t>(state) * elems);
+    float num = 0.f, den = 0.f;
+    for (size_t i = v0 + threadIdx.x; i < v1; i += kErrThreads) {
+        const float4 a = __ldcs(xv + i), b = __ldcs(rv + i);
+        const float d0 = a.x - b.x, d1 = a.y - b.y, d2 = a.z - b.z, d3 = a.w - b.w;
+        num += d0 * d0 + d1 * d1 + d2 * d2 + d3 * d3;
+        den += b.x * b.x + b.y * b.y + b.z * b.z + b.w * b.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        num += __shfl_xor_sync(0xffffffffu, num, o);
+        den += __shfl_xor_sync(0xffffffffu, den, o);
+    }
+    __shared__ float sn[kErrThreads / 32], sd[kErrThreads / 32];
+    if ((threadIdx.x & 31) == 0) { sn[threadIdx.x >> 5] = num; sd[threadIdx.x >> 5] = den; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float n = 0.f, d = 0.f;
+        for (int w = 0; w < kErrThreads / 32; ++w) { n += sn[w]; d += sd[w]; }
+        partials[2 * (static_cast<size_t>(state) * parts + part)] = n;
+        partials[2 * (static_cast<size_t>(state) * parts + part) + 1] = d;
+    }
+}
+
+__global__ void state_err_final_kernel(const float *__restrict__ partials, int parts, int n_states, float *__restrict__ rel_err) {
+    const int state = blockIdx.x * blockDim.x + threadIdx.x;
+    if (state >= n_states) return;
+    float n = 0.f, d = 0.f;
+    for (int p = 0; p < parts; ++p) {
+        n += partials[2 * (static_cast<size_t>(state) * parts + p)];
+        d += partials[2 * (static_cast<size_t>(state) * parts + p) + 1];
+    }
+    rel_err[state] = sqrtf(n) / sqrtf(d);
+}
+
+}  // namespace
+
+int state_err_parts(size_t elems) {
+    const size_t parts = (elems + kErrElemsPerCta - 1) / kErrElemsPerCta;
+    return static_cast<int>(parts < 1 ? 1 : (parts > 4096 ? 4096 : parts));
+}
+
+cudaError_t launch_state_rel_error(const float *x, const float *r, float *rel_err, int n_states, size_t elems,
+                                   float *partials, cudaStream_t s) {
+    const int parts = state_err_parts(elems);
+    state_err_partial_kernel<<<dim3(parts, n_states), kErrThreads, 0, s>>>(x, r, elems, parts, partials);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    state_err_final_kernel<<<(n_states + 127) / 128, 128, 0, s>>>(partials, parts, n_states, rel_err);
+    return cudaGetLastError();
+}
+
 }  // namespace lkv

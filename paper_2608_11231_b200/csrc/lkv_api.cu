@@ -249,6 +249,23 @@ int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, c
     return launch_mamba_logdecay(a, logdecay, s) == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
 }
 
+size_t lkv_state_rel_error_workspace_bytes(int n_states, size_t state_elems) {
+    if (n_states < 0 || state_elems == 0) return 0;
+    return align_up(sizeof(float) * 2 * static_cast<size_t>(n_states) * state_err_parts(state_elems) + 16, 256);
+}
+
+int lkv_state_rel_error(const float *S_init, const float *S_ref, float *rel_err, int n_states, size_t state_elems,
+                        void *workspace, size_t workspace_bytes, void *stream) {
+    if (n_states < 0 || state_elems == 0 || state_elems % 4 != 0 || n_states > 65535) return LKV_ERR_DIM;
+    if (n_states == 0) return LKV_OK;
+    if (!S_init || !S_ref || !rel_err) return LKV_ERR_NULL;
+    if (!aligned16(S_init) || !aligned16(S_ref) || !aligned16(workspace)) return LKV_ERR_ALIGN;
+    if (!workspace || workspace_bytes < lkv_state_rel_error_workspace_bytes(n_states, state_elems)) return LKV_ERR_WORKSPACE;
+    const cudaError_t e = launch_state_rel_error(S_init, S_ref, rel_err, n_states, state_elems,
+                                                 static_cast<float *>(workspace), static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
 int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
                 const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream) {
     if (!d) return LKV_ERR_NULL;

@@ -166,6 +166,23 @@ def test_artifact_producers_argument_errors(lib):
     assert y == b.LKV_ERR_NULL
 
 
+def test_state_rel_error_argument_errors(lib):
+    f = lambda a=FAKE, r=FAKE, out=FAKE, n=4, elems=1024, ws=FAKE, wsb=1 << 20: lib.lkv_state_rel_error(
+        a, r, out, n, elems, ws, wsb, None)
+    assert f(n=-1) == b.LKV_ERR_DIM
+    assert f(elems=0) == b.LKV_ERR_DIM
+    assert f(elems=1022) == b.LKV_ERR_DIM            # multiple of 4 for the 16-byte loads
+    assert f(n=0) == b.LKV_OK
+    assert f(a=None) == b.LKV_ERR_NULL
+    assert f(out=None) == b.LKV_ERR_NULL
+    assert f(r=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert f(ws=None) == b.LKV_ERR_WORKSPACE
+    assert f(wsb=16) == b.LKV_ERR_WORKSPACE
+    need = lib.lkv_state_rel_error_workspace_bytes(4, 1 << 20)
+    assert need >= 4 * 64 * 8 and need % 256 == 0    # 64 slices of 16384 floats per state, two sums each
+    assert lib.lkv_state_rel_error_workspace_bytes(4, 0) == 0
+
+
 def test_workspace_bytes(lib):
     d = _desc()
     small = b.lkv_workspace_bytes(b.LKV_WS_INIT, d, 1, 8)

@@ -114,3 +114,45 @@ def test_cache_building_pipeline_mamba_reproduces_the_full_prefix_state():
     S0 = host(b.lkv_init_state(states, lam, len(lens), b.LKV_INIT_EXACT, family=b.LKV_FAMILY_MAMBA2))
     _, S_ref = oracle.ssd_seq(cat["x"], cat["dt"], A, cat["B"], cat["C"])
     assert maxrel(S0, S_ref) <= TOL_BF16, maxrel(S0, S_ref)
+
+
+@pytest.mark.parametrize("n,shape", [(5, (2, 64, 64)), (3, (32, 128, 128)), (1, (4,))])
+def test_state_rel_error_matches_oracle(n, shape):
+    rng = np.random.default_rng(16)
+    ref = rng.standard_normal((n,) + shape).astype(np.float32)
+    init = (ref + 0.01 * rng.standard_normal(ref.shape)).astype(np.float32)
+    init[0] = ref[0]                                   # exact -> 0
+    if n > 1:
+        init[1] = 0.0                                  # empty-state initialiser -> 1
+    err = host(b.lkv_state_rel_error(dev(init), dev(ref)))
+    want = oracle.state_rel_error(init, ref)
+    assert err[0] == 0.0
+    assert np.abs(err - want).max() <= 1e-5 * max(1.0, want.max())
+    # whole layer as one state, and per head
+    one = host(b.lkv_state_rel_error(dev(init), dev(ref), n_states=1))
+    assert abs(one[0] - oracle.state_rel_error(init, ref, n_states=1)[0]) <= 1e-5
+    if len(shape) == 3:
+        per_head = host(b.lkv_state_rel_error(dev(init), dev(ref), n_states=n * shape[0]))
+        assert np.abs(per_head - oracle.state_rel_error(init, ref, n_states=n * shape[0])).max() <= 1e-5
+
+
+def test_state_rel_error_of_the_two_initialisers():
+    """The paper's diagnostic on the library's own initialisers: exact composition sits at the rounding floor,
+    the last-block state differs from the full-prefix state by the carried part."""
+    torch = _t()
+    bf = torch.bfloat16
+    H_k, H_v, d, lens = 2, 4, 128, [256, 256, 256]
+    rng = np.random.default_rng(17)
+    chunks = [wl.gdn_tokens(rng, L, H_k, H_v, d, d, live_chunk_len=256) for L in lens]
+    cat = _cat(chunks, ("q", "k", "v", "g", "beta"))
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    q, k, v, g, beta = dev(cat["q"], bf), dev(cat["k"], bf), dev(cat["v"], bf), dev(cat["g"]), dev(cat["beta"])
+    _, states = b.lkv_gdn_fwd(q, k, v, g, beta, cu_seqlens=cu, want_outputs=False)
+    trans = b.lkv_gdn_chunk_transition(k, g, beta, cu_seqlens=cu)
+    S_ex = b.lkv_init_state(states, trans, 3, b.LKV_INIT_EXACT, family=b.LKV_FAMILY_GDN)
+    S_lb = b.lkv_init_state(states, None, 3, b.LKV_INIT_LAST, family=b.LKV_FAMILY_GDN)
+    S_star = dev(oracle.gdn_seq(cat["q"], cat["k"], cat["v"], cat["g"], cat["beta"])[1].astype(np.float32))
+    e_ex = host(b.lkv_state_rel_error(S_ex, S_star, n_states=1))[0]
+    e_lb = host(b.lkv_state_rel_error(S_lb, S_star, n_states=1))[0]
+    assert e_ex <= 2e-2 and e_lb > 5 * e_ex
+

@@ -372,3 +372,25 @@ def test_generators_are_seeded_and_shaped():
     assert [r["family"] for r in reqs].count("gdn") == 32
     assert np.array_equal(wl.request_permutation(3, 0, 32), np.arange(32))
     assert sorted(wl.request_permutation(3, 5, 32).tolist()) == list(range(32))
+
+
+def test_state_rel_error_closed_forms():
+    """Section 3.2 diagnostic: values fixed by hand, not by the formula's own code."""
+    ref = np.zeros((3, 2, 4))
+    ref[0, 0, 0] = 3.0
+    ref[0, 1, 3] = 4.0          # ||ref_0|| = 5
+    ref[1] = 1.0                # ||ref_1|| = sqrt(8)
+    ref[2, 1, 1] = 2.0
+    init = ref.copy()
+    init[0, 0, 1] = 5.0         # one entry off by 5 -> 5 / 5
+    init[1] *= 1.5              # scaled copy -> |1.5 - 1|
+    init[2] = 0.0               # the "empty state" initialiser -> exactly 1
+    err = oracle.state_rel_error(init, ref)
+    assert np.allclose(err, [1.0, 0.5, 1.0], rtol=0, atol=1e-15)
+    assert oracle.state_rel_error(ref, ref).tolist() == [0.0, 0.0, 0.0]
+    # one number for the whole array = ratio of the norms of the concatenated vectors
+    whole = oracle.state_rel_error(init, ref, n_states=1)
+    assert np.isclose(whole[0], np.sqrt(25.0 + 8 * 0.25 + 4.0) / np.sqrt(25.0 + 8.0 + 4.0), rtol=1e-15)
+    # sign and order of the arguments matter only through the denominator
+    assert np.isclose(oracle.state_rel_error(ref[:1], init[:1])[0], 5.0 / np.sqrt(50.0), rtol=1e-15)
+
