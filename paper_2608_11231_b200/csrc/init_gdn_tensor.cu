@@ -6,8 +6,9 @@
 //   - S^T (128 state columns = TMEM lanes, 128 state rows = TMEM columns, fp32 read as tf32) is the
 //     A operand of tcgen05.mma, taken straight from TMEM;
 //   - T_j, row-major fp32 as cached, is exactly the K-major B operand; a producer warp streams it
-//     (and the S_j tiles) through shared memory with TMA and pulls later chunks into L2 ahead of
-//     time, and a separate warp issues the MMAs, so neither waits for the other's instructions;
+//     (and the S_j tiles) through shared memory with TMA, and a separate warp issues the MMAs, so
+//     neither waits for the other's instructions.  (No L2 prefetch of later chunks: with one CTA per
+//     SM the prefetched lines were evicted before their use and DRAM traffic grew by half.)
 //   - D = S^T T_j^T lands in a TMEM accumulator in two 64-column halves; two epilogue warpgroups
 //     (thread = one state column, warpgroup = one half of the state rows) add S_j^T, round, and
 //     store the result as the next step's A operand (double-buffered in TMEM), the first half
@@ -29,7 +30,6 @@ constexpr int kD = 128;                      // d_k = d_v = MMA M = MMA N (two h
 constexpr int kTStageBytes = kD * kD * 4;    // one transition: 4 K-blocks of [128 rows x 128 B]
 constexpr int kStages = 2;                   // transitions in the shared-memory ring
 constexpr int kSHalfBytes = 64 * kD * 4;     // half of a cached state: 4 column blocks of [64 rows x 128 B]
-constexpr int kLook = 5;                     // L2 look-ahead, in chain steps
 constexpr int kEpiThreads = 256;             // two epilogue warpgroups
 constexpr int kThreads = kEpiThreads + 64;   // + MMA warp + TMA warp
 constexpr int kSmemBytes = kStages * kTStageBytes + 2 * kSHalfBytes + 1024;
@@ -103,21 +103,15 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
                 for (int cb = 0; cb < 4; ++cb)
                     tma_load_2d(sS + half * kSHalfBytes + cb * 64 * 128, &mapS, cb * 32, prow(j) + 64 * half, &bar_fullS[half]);
             };
-            auto prefetch = [&](int j) {
-                for (int kb = 0; kb < 4; ++kb) tma_prefetch_l2_2d(&mapT, kb * 32, prow(j));
-                for (int q = 0; q < 8; ++q) tma_prefetch_l2_2d(&mapS, (q & 3) * 32, prow(j) + 64 * (q >> 2));
-            };
             load_S(0, 0);
             load_S(0, 1);
             for (int j = 1; j < K && j <= kStages; ++j) load_T(j);
-            for (int j = 1; j < K && j <= kLook; ++j) prefetch(j);
             for (int j = 1; j < K; ++j) {
                 // T_{j+1} takes over the stage of T_{j-1} as soon as the MMAs of step j-1 are done
                 if (j >= 2 && j + 1 < K) {
                     mbar_wait(&bar_freeT[stage_of(j - 1)], phase_of(j - 1), &dead, a.status);
                     load_T(j + 1);
                 }
-                if (j + kLook < K) prefetch(j + kLook);
                 // S_j takes over the tile halves as the epilogue of step j-1 lets go of them
                 for (int half = 0; half < 2; ++half) {
                     mbar_wait(&bar_freeS[half], (j - 1) & 1, &dead, a.status);
