@@ -60,9 +60,10 @@ def ssd_scan_flops(tokens: int, s=SSD_SHAPE, Q=SSD_BLOCK) -> float:
     return (2.0 * (2 * s["N"] * s["P"] + Q * s["P"]) * s["H"] + 2.0 * Q * s["N"] * s["G"]) * tokens
 
 
-# DRAM bytes (read + write) per scanned token from the ncu capture of one 16384-token launch of each scan kernel
-# (8 sequences x 2048 tokens); the traffic of a scan grows in proportion to its tokens.
-NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.03e6 + 119.80e6) / 16384, "mamba2.scan": None}
+# DRAM bytes (read + write) per scanned token from ncu captures of one launch of each scan kernel (GDN: 8 sequences x
+# 2048 tokens; Mamba-2: 16 sequences x 4096 tokens, initial and final states included); the traffic of a scan grows
+# in proportion to its tokens.
+NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.69e6 + 119.74e6) / 16384, "mamba2.scan": (788.81e6 + 671.33e6) / 65536}
 
 
 def gdn_scan_bytes(tokens: int, s=GDN_SHAPE) -> float:
@@ -401,7 +402,7 @@ def run_ours(args):
         per_token = NCU_DRAM_BYTES_PER_TOKEN.get(dom)
         roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
                     traffic=None if per_token is None else per_token * f.scan_tokens,
-                    traffic_source="ncu dram bytes of a 16384-token launch, scaled by tokens", kernel=dom,
+                    traffic_source="ncu dram bytes of a smaller launch of the same kernel, scaled by tokens", kernel=dom,
                     peak_source=peak_src)
     else:
         nbytes = f.pool_bytes_unique + f.S0.numel() * 4
