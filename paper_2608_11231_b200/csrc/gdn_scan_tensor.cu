@@ -21,7 +21,8 @@
 // (2) -> r -> (3) -> U o w -> (5) -> state copy.
 // A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
 // Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 out,
-// 12-15 prep (the inverse), 16 TMA loads, 17 MMA issue, 18 TMA store of the output tile, 19 per-block scalars
+// 12-15 prep (the inverse), 16 TMA loads and the store of the output tile, 17 MMA issue of the chain ((2), (3), (5)),
+// 18 MMA issue of the prep side ((1), (6)), 19 per-block scalars
 // (running up to three blocks ahead).  All waits on mbarriers are bounded.
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -68,7 +69,7 @@ struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
     uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done, o_free[2];
     // 128-thread barriers (prep or out warpgroup)
-    uint64_t m_ready[2], o_done[4], inv_done[2], o_staged;
+    uint64_t m_ready[2], o_done[4], inv_done[2], o_staged[2];
     // 64-thread barriers (the two halves of the out warpgroup)
     uint64_t a_ready, p_ready, gb_ready[4], mpm_ready[2];
     // 256-thread barriers (both chain warpgroups)
@@ -206,7 +207,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         uint64_t *b1 = &bars.full_qk[0];
         for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
         uint64_t *b128 = &bars.m_ready[0];
-        for (int i = 0; i < 9; ++i) mbar_init(b128 + i, 128);
+        for (int i = 0; i < 10; ++i) mbar_init(b128 + i, 128);
         uint64_t *b64 = &bars.a_ready;
         for (int i = 0; i < 8; ++i) mbar_init(b64 + i, (i >= 2 && i < 6) ? 32 : 64);   // gb_ready: the scalar warp
         uint64_t *b256 = &bars.v_free;
@@ -226,6 +227,18 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tma_prefetch_desc(&mapQ);
             tma_prefetch_desc(&mapK);
             if (a.v) tma_prefetch_desc(&mapV);
+            if (a.o) tma_prefetch_desc(&mapO);
+            // the output tile of block b (whole blocks only) leaves its staging buffer, the [M; PM] buffer of parity b
+            auto store_o = [&](int b) {
+                mbar_wait(&bars.o_staged[b & 1], (b >> 1) & 1, &dead, a.status);
+                const int t0 = t_begin + b * kC;
+                if (a.o && t0 + kC <= t_end && !dead) {
+                    tma_store_2d(&mapO, sm + kOffMPM + (b & 1) * (kD * 128), h * kD, t0);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+                mbar_arrive(&bars.o_free[b & 1]);
+            };
             for (int b = 0; b < nblk; ++b) {
                 const int st = b & 1;
                 const int row = t_begin + b * kC;
@@ -249,7 +262,12 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     mbar_expect_tx(&bars.full_v, kC * kD * 2);
                     tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
                 }
+                // the output of block b-2 was staged about one block ago; the inverse of block b needs its buffer only later
+                if (b >= 2) store_o(b - 2);
             }
+            if (nblk >= 2) store_o(nblk - 2);
+            store_o(nblk - 1);
+            tma_store_wait_all();
         }
     } else if (warp == 19) {
         // ======================================================= scalar warp: lane = tokens 2 lane, 2 lane + 1 of the block
@@ -301,31 +319,10 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_arrive(&bars.gb_ready[b & 3]);
         }
     } else if (warp == 18) {
-        // ======================================================= TMA store of the output tiles (whole blocks only)
-        if (lane == 0) {
-            if (a.o) tma_prefetch_desc(&mapO);
-            for (int b = 0; b < nblk; ++b) {
-                mbar_wait(&bars.o_staged, b & 1, &dead, a.status);
-                const int t0 = t_begin + b * kC;
-                if (a.o && t0 + kC <= t_end && !dead) {
-                    tma_store_2d(&mapO, sm + kOffMPM + (b & 1) * (kD * 128), h * kD, t0);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
-                mbar_arrive(&bars.o_free[b & 1]);
-            }
-            tma_store_wait_all();
-        }
-    } else if (warp == 17) {
-        // ======================================================= MMA issuer (one elected thread, tight code)
+        // ======================================================= second MMA issuer: (1) and (6), the prep side
         if (elect_one()) {
             constexpr uint32_t idG = umma_idesc(kFmtBF16, false, false, 128, 64);    // (1)
-            constexpr uint32_t idD1 = umma_idesc(kFmtBF16, false, false, 128, 128);  // (2), (3)
             constexpr uint32_t idPM = umma_idesc(kFmtBF16, false, true, 128, 64);    // (6): B = M read MN-major
-            constexpr uint32_t idDS = umma_idesc(kFmtBF16, false, true, 128, 128);   // (5): B = K tile read MN-major
-            const uint64_t dSt = umma_desc(smem_u32(sm + kOffSt), 0, 1024);
-            const uint64_t dR = umma_desc(smem_u32(sm + kOffR), 0, 1024);
-            const uint64_t dUw = umma_desc(smem_u32(sm + kOffUw), 0, 1024);
             const uint64_t dP = umma_desc(smem_u32(sm + kOffP - kC * 128), 0, 1024);
             const uint64_t dMPM0 = umma_desc(smem_u32(sm + kOffMPM), 0, 1024);
             auto issue_G = [&](int b) {
@@ -337,53 +334,55 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
                 umma_commit(&bars.g_done);
             };
-            auto issue_PM = [&](int b) {   // PM = P M: A = P (K = i), B = M rows of the [M; PM] tile read MN-major
-                const uint64_t dM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
-#pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmPM, dP + 2 * k, dM + ((k * 16 * 128) >> 4), idPM, k > 0);
-                umma_commit(&bars.pm_done);
-            };
             mbar_wait(&bars.full_qk[0], 0, &dead, a.status);
             tc_fence_after_sync();
             issue_G(0);
             for (int b = 0; b < nblk; ++b) {
                 const uint32_t par = b & 1;
-                const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
-                // Three MMAs of this iteration have independent inputs and are issued in the order their inputs arrive
-                // (a blocking wait for one would hold back the others):
-                //   (6) of block b:   the inverse (m_ready) and P (p_ready);
-                //   (2) of block b:   the bf16 state copy (st_ready) and the D1 / UP accumulators drained (o_done of b-1);
-                //   (1) of block b+1: the G columns drained by the mask epilogue of block b, and the next Q / K tiles.
-                uint32_t pending = 4u | 1u | (b + 1 < nblk ? 2u : 0u);
-                for (uint32_t spins = 0; pending != 0;) {
-                    if ((pending & 4u) && mbar_test_wait(&bars.m_ready[b & 1], (b >> 1) & 1) && mbar_test_wait(&bars.p_ready, par)) {
-                        tc_fence_after_sync();
-                        issue_PM(b);
-                        pending &= ~4u;
-                    } else if ((pending & 1u) && mbar_test_wait(&bars.st_ready, par) &&
-                               (b == 0 || mbar_test_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1))) {
-                        tc_fence_after_sync();
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const uint64_t offA = ((k >> 2) * (kD * 128) + (k & 3) * 32) >> 4;
-                            const uint64_t offB = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
-                            umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
-                        }
-                        umma_commit(&bars.d1_done);
-                        pending &= ~1u;
-                    } else if ((pending & 2u) && mbar_test_wait(&bars.a_ready, par) && mbar_test_wait(&bars.p_ready, par) &&
-                               mbar_test_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1)) {
-                        tc_fence_after_sync();
-                        issue_G(b + 1);
-                        pending &= ~2u;
-                    } else if (++spins > kSpinLimit || dead) {
-                        if (!dead) {
-                            dead = 1;
-                            if (a.status) atomicExch(a.status, 1);
-                        }
-                        break;
-                    }
+                // (1) of the next block as soon as the mask epilogue of this one has drained the G columns
+                if (b + 1 < nblk) {
+                    mbar_wait(&bars.a_ready, par, &dead, a.status);
+                    mbar_wait(&bars.p_ready, par, &dead, a.status);
+                    mbar_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+                    issue_G(b + 1);
                 }
+                // (6) of this block as soon as its inverse is there: PM = P M, A = P (K = i), B = M rows of [M; PM] read MN-major
+                mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+                mbar_wait(&bars.p_ready, par, &dead, a.status);
+                // the accumulator of (6) must have been read for block b-1 (its PM rows are in the operand)
+                if (b >= 1) mbar_wait(&bars.mpm_ready[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
+                tc_fence_after_sync();
+                const uint64_t dM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmPM, dP + 2 * k, dM + ((k * 16 * 128) >> 4), idPM, k > 0);
+                umma_commit(&bars.pm_done);
+            }
+        }
+    } else if (warp == 17) {
+        // ======================================================= first MMA issuer: (2), (3), (5), the block-to-block chain
+        if (elect_one()) {
+            constexpr uint32_t idD1 = umma_idesc(kFmtBF16, false, false, 128, 128);  // (2), (3)
+            constexpr uint32_t idDS = umma_idesc(kFmtBF16, false, true, 128, 128);   // (5): B = K tile read MN-major
+            const uint64_t dSt = umma_desc(smem_u32(sm + kOffSt), 0, 1024);
+            const uint64_t dR = umma_desc(smem_u32(sm + kOffR), 0, 1024);
+            const uint64_t dUw = umma_desc(smem_u32(sm + kOffUw), 0, 1024);
+            const uint64_t dMPM0 = umma_desc(smem_u32(sm + kOffMPM), 0, 1024);
+            for (int b = 0; b < nblk; ++b) {
+                const uint32_t par = b & 1;
+                const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
+                // (2) needs the bf16 state copy of block b, the D1 / UP accumulators drained, and the Q / K tiles
+                mbar_wait(&bars.st_ready, par, &dead, a.status);
+                if (b > 0) mbar_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1, &dead, a.status);
+                mbar_wait(&bars.full_qk[b & 1], (b >> 1) & 1, &dead, a.status);
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint64_t offA = ((k >> 2) * (kD * 128) + (k & 3) * 32) >> 4;
+                    const uint64_t offB = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
+                    umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
+                }
+                umma_commit(&bars.d1_done);
                 // (3) [U | PU] = R^T [M; PM]^T
                 mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
                 mbar_wait(&bars.r_ready, par, &dead, a.status);
@@ -618,7 +617,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             }
             tc_fence_before_sync();
             mbar_arrive(&bars.o_done[b & 3]);
-            mbar_arrive(&bars.o_staged);
+            mbar_arrive(&bars.o_staged[b & 1]);
         }
     } else {
         // ======================================================= chain warpgroups: lane = state column j, `half` = token / row half
