@@ -398,3 +398,32 @@ def test_scans_with_violent_decay_take_the_exact_exponent_path():
     y, hT = _run_ssd(st, A, rng.standard_normal((1, H, N, P)).astype(np.float32) * 0 + 1.0, "bf16")
     y_ref, hT_ref = oracle.ssd_seq(st["x"], st["dt"], A, st["B"], st["C"], np.ones((H, N, P)))
     assert maxrel(y, y_ref) <= TOL_BF16 and maxrel(hT[0], hT_ref) <= TOL_BF16
+
+
+def test_scans_with_more_sequences_than_fit_the_parameter_block():
+    """1100 short sequences: cu_seqlens no longer fits the kernel parameter block and travels through the
+    workspace.  Every sequence's final state and a sample of outputs are checked against the oracle."""
+    torch = _torch()
+    bf = torch.bfloat16
+    rng = np.random.default_rng(31)
+    n_seq = 1100
+    lens = rng.integers(0, 40, size=n_seq)
+    lens[[5, 500, 1099]] = [130, 70, 200]          # a few that span several blocks
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T = int(cu[-1])
+    g = wl.gdn_tokens(rng, T, 1, 2, 128, 128)
+    o, ST = b.lkv_gdn_fwd(dev(g["q"], bf), dev(g["k"], bf), dev(g["v"], bf), dev(g["g"]), dev(g["beta"]), cu_seqlens=cu)
+    o, ST = host(o), host(ST)
+    m = wl.ssd_tokens(rng, T, 2, 64, 128, 1)
+    A = wl.ssd_A(rng, 2)
+    y, MT = b.lkv_ssd_fwd(dev(m["x"], bf), dev(m["dt"]), dev(A), dev(m["B"], bf), dev(m["C"], bf), cu_seqlens=cu)
+    y, MT = host(y), host(MT)
+    for s in [0, 5, 499, 500, 777, 1098, 1099] + list(rng.integers(0, n_seq, size=8)):
+        a0, a1 = int(cu[s]), int(cu[s + 1])
+        if a1 == a0:
+            assert not ST[s].any() and not MT[s].any()
+            continue
+        o_ref, S_ref = oracle.gdn_seq(*[g[n][a0:a1] for n in ("q", "k", "v", "g", "beta")])
+        assert maxrel(o[a0:a1], o_ref) <= TOL_BF16 and maxrel(ST[s], S_ref) <= TOL_BF16
+        y_ref, M_ref = oracle.ssd_seq(m["x"][a0:a1], m["dt"][a0:a1], A, m["B"][a0:a1], m["C"][a0:a1])
+        assert maxrel(y[a0:a1], y_ref) <= TOL_BF16 and maxrel(MT[s], M_ref) <= TOL_BF16
