@@ -344,11 +344,19 @@ def run_ours(args):
         for f in fams:
             f.step()
 
+    e2e_streams = [torch.cuda.Stream() for _ in fams]
+
     def step_e2e():
-        for f in fams:
-            f.upload()
-            f.step()
-            f.download()
+        # one stream per family: the device->host copies of one overlap the host->device copies of the other
+        cur = torch.cuda.current_stream()
+        for f, st in zip(fams, e2e_streams):
+            st.wait_stream(cur)
+            with torch.cuda.stream(st):
+                f.upload()
+                f.step()
+                f.download()
+        for st in e2e_streams:
+            cur.wait_stream(st)
 
     # clocks are sampled from the warm-up to the end of the end-to-end steps: the GPU is busy throughout
     sampler = ClockSampler(local)
