@@ -165,6 +165,36 @@ class Family:
         self.init_exact()
         self.scan()
 
+    def make_full_prefill(self, tokens: int):
+        """One request's whole context as one sequence (device-generated stand-in tokens, timing only): the scan of
+        it from the empty state is the full-prefill reference that the initialisers + recompute scan replace."""
+        torch, bf = self.torch, self.torch.bfloat16
+        gen = torch.Generator(device="cuda").manual_seed(5)
+        rn = lambda *shape: torch.randn(shape, generator=gen, device="cuda")
+        if self.fam == "gdn":
+            s = GDN_SHAPE
+            nrm = torch.nn.functional.normalize
+            self.full = dict(q=nrm(rn(tokens, s["H_k"], s["d_k"]), dim=-1).to(bf), k=nrm(rn(tokens, s["H_k"], s["d_k"]), dim=-1).to(bf),
+                             v=rn(tokens, s["H_v"], s["d_v"]).to(bf), g=-0.1 * torch.nn.functional.softplus(rn(tokens, s["H_v"])),
+                             beta=torch.sigmoid(rn(tokens, s["H_v"])))
+            self.full_ST = torch.empty((1,) + self.state_shape, dtype=torch.float32, device="cuda")
+            self.full_out = torch.empty((tokens, s["H_v"], s["d_v"]), dtype=bf, device="cuda")
+        else:
+            s = SSD_SHAPE
+            self.full = dict(x=rn(tokens, s["H"], s["P"]).to(bf), dt=torch.nn.functional.softplus(-2.0 + 0.5 * rn(tokens, s["H"])),
+                             B=(rn(tokens, s["G"], s["N"]) / s["N"] ** 0.5).to(bf), C=(rn(tokens, s["G"], s["N"]) / s["N"] ** 0.5).to(bf))
+            self.full_ST = torch.empty((1,) + self.state_shape, dtype=torch.float32, device="cuda")
+            self.full_out = torch.empty((tokens, s["H"], s["P"]), dtype=bf, device="cuda")
+        self.full_tokens = tokens
+
+    def full_prefill(self):
+        b, d = self.b, self.full
+        if self.fam == "gdn":
+            b.lkv_gdn_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], None, self.full_out, self.full_ST, workspace_t=self.ws_scan)
+        else:
+            b.lkv_ssd_fwd(d["x"], d["dt"], self.dev["A"], d["B"], d["C"], None, self.full_out, self.full_ST,
+                          workspace_t=self.ws_scan)
+
 
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons every 200 ms while the timed region runs."""
@@ -380,6 +410,17 @@ def run_ours(args):
     e2e_steps = max(1, min(args.steps, 3))
     step_e2e()
     ms_e2e = timed_back_to_back(step_e2e, e2e_steps)
+    # full-prefill reference (single-family configurations): one request's whole context scanned from the empty state
+    full = {}
+    if args.workload in ("cfg1", "cfg2", "cfg3"):
+        for f in fams:
+            f.make_full_prefill(f.reqs[0]["total"])
+            g = graph_of(f.full_prefill)
+            t = timed_flushed(g.replay, max(args.steps, 5), reduce="median")
+            # the same request served from the cache: its share of the batched init calls plus its recompute scan
+            t_cached = (parts[f"{f.fam}.init_exact"] + parts[f"{f.fam}.scan"]) / f.n_req
+            full[f.fam] = dict(tokens=f.full_tokens, us=1e3 * t, tokens_per_s=f.full_tokens / (t * 1e-3),
+                               cached_path_us_per_request=1e3 * t_cached, cached_over_full=t_cached / t)
     clocks = sampler.stop() if rank == 0 else None
 
     if world > 1:
@@ -446,6 +487,8 @@ def run_ours(args):
         gpu_launches=sum(f.launches for f in fams) * args.steps,
         scan_tokens_per_s=job_scan_tokens / (ms * 1e-3),
         roofline=roof, kernels=detail, clocks=clocks)
+    if full:
+        line["full_prefill"] = full
     if base is not None:
         line["cpu_baseline"] = base
     print(json.dumps(line))
