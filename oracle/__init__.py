@@ -18,6 +18,8 @@ Functions and the passage of the paper each one states:
 ``init_exact_mamba``   Eq. 6 with scalar transitions
 ``init_single``        the single-block initialiser S_init = S_b (Section 3.2,
                        "Single-block initialization"; Appendix A for b != K)
+``state_rel_error``    the per-state relative error ||S_init - S*|| / ||S*|| of
+                       Section 3.2, "Diagnosis via relative error" (numpy)
 
 Parity status: every function above is pinned by the CPU tests (brute force on
 the concatenated prefix, literal Eq. 3 matrices, closed forms and library
