@@ -360,6 +360,13 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
         const int half = warp >> 2;
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         __nv_bfloat16 *y = static_cast<__nv_bfloat16 *>(a.y);
+        {
+            // operand columns above the diagonal for every row of this warp are never written again: zero them once
+            const uint32_t z[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            for (int q = 0; q < 4; ++q)
+                if (64 * half + 16 * q > 32 * (warp & 3) + 31) tmem_st8(lane_base + kTmGp + 32 * half + 8 * q, z);
+            tmem_st_wait();
+        }
         for (int b = 0; b < nblk; ++b) {
             const float *sc = scal + (b % 3) * kScFloats;
             mbar_wait(&bars.sc_ready[b % 3], (b / 3) & 1, &dead, a.status);
@@ -375,10 +382,11 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 const bool fast = sc[5 * kQ] == 0.f;
 #pragma unroll 1
                 for (int q = 0; q < 4; ++q) {
+                    const int i0 = 64 * half + 16 * q;
+                    if (i0 > 32 * (warp & 3) + 31) break;   // above the diagonal for every row of this warp: stays zero
                     uint32_t rr[16];
                     tmem_ld16(lane_base + kTmG + 64 * half + 16 * q, rr);
                     tmem_ld_wait();
-                    const int i0 = 64 * half + 16 * q;
                     uint32_t w[8];
                     if (fast) {
                         float aa;
