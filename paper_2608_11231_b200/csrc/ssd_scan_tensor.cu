@@ -391,15 +391,25 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                     if (fast) {
                         float aa;
                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(lt - sc[i0], 0.f)));
+                        if (i0 + 15 <= 32 * (warp & 3)) {
+                            // the whole group lies below the diagonal for every row of this warp: no masking
 #pragma unroll
-                        for (int c = 0; c < 16; c += 4) {
-                            const float4 f = *reinterpret_cast<const float4 *>(sc + 3 * kQ + i0 + c);
-                            const float v0 = (i0 + c <= t) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
-                            const float v1 = (i0 + c + 1 <= t) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
-                            const float v2 = (i0 + c + 2 <= t) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
-                            const float v3 = (i0 + c + 3 <= t) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
-                            w[c / 2] = pack_bf16(v0, v1);
-                            w[c / 2 + 1] = pack_bf16(v2, v3);
+                            for (int c = 0; c < 16; c += 4) {
+                                const float4 f = *reinterpret_cast<const float4 *>(sc + 3 * kQ + i0 + c);
+                                w[c / 2] = pack_bf16(__uint_as_float(rr[c]) * aa * f.x, __uint_as_float(rr[c + 1]) * aa * f.y);
+                                w[c / 2 + 1] = pack_bf16(__uint_as_float(rr[c + 2]) * aa * f.z, __uint_as_float(rr[c + 3]) * aa * f.w);
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 16; c += 4) {
+                                const float4 f = *reinterpret_cast<const float4 *>(sc + 3 * kQ + i0 + c);
+                                const float v0 = (i0 + c <= t) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                                const float v1 = (i0 + c + 1 <= t) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                                const float v2 = (i0 + c + 2 <= t) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                                const float v3 = (i0 + c + 3 <= t) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                                w[c / 2] = pack_bf16(v0, v1);
+                                w[c / 2 + 1] = pack_bf16(v2, v3);
+                            }
                         }
                     } else {
 #pragma unroll
