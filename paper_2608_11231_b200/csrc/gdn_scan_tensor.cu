@@ -527,24 +527,38 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 const float coef = (x < kC) ? 1.f : sc[kC + t];     // rows of P: 1, rows of A: beta_t
                 const int lim = (x < kC) ? t : t - 1;               // P keeps the diagonal, A is strictly lower
                 const bool fast = sc[5 * kC] + sc[5 * kC + 1] == 0.f;
+                const int row_hi = (t & 32) + 31;   // last row (token) of this warp
 #pragma unroll 1
                 for (int q = 0; q < 4; ++q) {
+                    const int i0 = 16 * q;
+                    if (i0 > row_hi) break;   // above the diagonal for every row of this warp: zeroed once, never written
                     uint32_t rr[16];
                     tmem_ld16(lane_base + kTmG + 16 * q, rr);
                     tmem_ld_wait();
-                    const int i0 = 16 * q;
                     float v[16];
                     if (fast) {
                         float aa;
                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(cgt - sc[i0], 0.f)));
                         aa *= coef;
+                        if (i0 + 15 <= row_hi - 32) {
+                            // below the diagonal for every row of this warp: no masking
 #pragma unroll
-                        for (int c = 0; c < 16; c += 4) {
-                            const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                            v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
-                            v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
-                            v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
-                            v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                            for (int c = 0; c < 16; c += 4) {
+                                const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                                v[c] = __uint_as_float(rr[c]) * aa * f.x;
+                                v[c + 1] = __uint_as_float(rr[c + 1]) * aa * f.y;
+                                v[c + 2] = __uint_as_float(rr[c + 2]) * aa * f.z;
+                                v[c + 3] = __uint_as_float(rr[c + 3]) * aa * f.w;
+                            }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 16; c += 4) {
+                                const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                                v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                                v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                                v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                                v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                            }
                         }
                     } else {
 #pragma unroll
@@ -569,6 +583,23 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             }
             if (pm_pending) pm_rows(b - 1);
         };
+        if ((x & 32) == 0) {
+            // columns 32..63 of rows 0..31 lie above the diagonal in P and in both A buffers: zero them once
+            const int t = x & 63;
+            float z[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) z[c] = 0.f;
+            for (int q = 2; q < 4; ++q) {
+                if (x < kC) {
+                    store_row_chunks(sm + kOffP, t, 2 * q, z);
+                } else {
+                    for (int bufi = 0; bufi < 2; ++bufi)
+                        for (int c = 0; c < 16; c += 4)
+                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sm + kOffA) + bufi * (kC * kLd) + t * kLd + 16 * q + c) =
+                                make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
         g_epilogue(0);
         for (int b = 0; b < nblk; ++b) {
             if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
