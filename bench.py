@@ -231,14 +231,14 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def cpu_baseline_sample(pairs: int = 8):
+def cpu_baseline_sample(pairs: int = 8, T: int = 12288):
     """The oracle as it stands, timed on this machine's cores on a bounded sample of the workload:
-    `pairs` times, exact composition of one GDN request (K = 16) plus a 12288-token GDN scan, all 32 value
-    heads, and the same for one Mamba-2 request (K = 16, 12288 tokens, 80 heads)."""
+    `pairs` times, exact composition of one GDN request (K = 16) plus a T-token GDN scan, all 32 value
+    heads, and the same for one Mamba-2 request (K = 16, T tokens, 80 heads)."""
     import oracle
     rng = np.random.default_rng(99)
     s, m = GDN_SHAPE, SSD_SHAPE
-    T, K = 12288, 16
+    K = 16
     tok = wl.gdn_tokens(rng, T, s["H_k"], s["H_v"], s["d_k"], s["d_v"])
     states = wl.synthetic_states(rng, K, s["H_v"], s["d_k"], s["d_v"])
     trans = wl.cheap_gdn_transitions(rng, K, s["H_v"], s["d_k"])
@@ -473,6 +473,16 @@ def run_ours(args):
             compose_frac_of_hbm=comp_bytes / (parts[f"{f.fam}.init_exact"] * 1e-3) / 1e9 / peaks["hbm_gbs"])
 
     base, _ = cpu_baseline_sample() if world == 1 else (None, None)
+    if base is not None:
+        # the same oracle on one thread, on a quarter-size sample (about as long as the all-core run)
+        import oracle
+        n_all = oracle.num_threads()
+        oracle.set_num_threads(1)
+        try:
+            one, _ = cpu_baseline_sample(pairs=1, T=3072)
+        finally:
+            oracle.set_num_threads(n_all)
+        base["one_thread"] = dict(value=one["value"], sample=one["sample"])
     line = dict(
         metric=METRIC, value=job_context_tokens / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
         warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -549,10 +559,11 @@ def run_sweep(args):
                     e1.synchronize()
                     ts.append(e0.elapsed_time(e1) * 1e3)
                 us = statistics.median(ts)
+                p90 = sorted(ts)[min(len(ts) - 1, int(0.9 * len(ts)))]
                 nbytes = (states.numel() + S0.numel()) * 4 + trans.numel() * 4
                 if fam == "gdn":   # the first chunk's transition is never read
                     nbytes -= n_req * H * dk * dk * 4
-                rows.append(dict(family=fam, requests=n_req, K=K, us=round(us, 2), gbs=round(nbytes / us / 1e3, 1),
+                rows.append(dict(family=fam, requests=n_req, K=K, us=round(us, 2), p90_us=round(p90, 2), gbs=round(nbytes / us / 1e3, 1),
                                  frac_of_hbm=round(nbytes / us / 1e3 / hbm, 3)))
                 del states, trans, S0
     print(json.dumps(dict(sweep="compose_us_vs_K", timing="graph replay of one launch between CUDA events (includes "
