@@ -89,7 +89,7 @@ bool init_mamba_stream_supported(const InitArgs &a, bool pool_bf16);
 cudaError_t launch_init_mamba_exact_stream(const InitArgs &a, cudaStream_t s);
 cudaError_t launch_init_gdn_exact_fp32(const InitArgs &a, bool pool_bf16, cudaStream_t s);
 bool init_gdn_exact_tensor_supported(const InitArgs &a, bool pool_bf16);
-cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, cudaStream_t s);
+cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, bool pool_bf16, cudaStream_t s);
 
 bool gdn_scan_fp32_supported(int d_k, int d_v);
 cudaError_t launch_gdn_scan_fp32(const GdnArgs &a, bool io_bf16, cudaStream_t s);

@@ -54,12 +54,16 @@ __device__ __forceinline__ void umma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, u
 __device__ __forceinline__ int stage_of(int j) { return (j - 1) % kStages; }
 __device__ __forceinline__ uint32_t phase_of(int j) { return static_cast<uint32_t>((j - 1) / kStages) & 1u; }
 
+// SBF16: the cached states are stored as bf16 (the transitions are fp32 either way); S0 is written as fp32.
+template <bool SBF16>
 __global__ void __launch_bounds__(kThreads, 1)
 init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_constant__ CUtensorMap mapT,
                              const __grid_constant__ CUtensorMap mapS) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char *sS = sm + kStages * kTStageBytes;   // [half][column block][64 rows][32 floats]
+    // fp32 pool: [half][4 column blocks][64 rows][32 floats]; bf16 pool: [half][2 column blocks][64 rows][64 bf16]
+    unsigned char *sS = sm + kStages * kTStageBytes;
+    constexpr int kSHalf = SBF16 ? kSHalfBytes / 2 : kSHalfBytes;   // bytes of half a cached state in the pool's dtype
     __shared__ uint64_t bar_fullT[kStages], bar_freeT[kStages], bar_fullS[2], bar_freeS[2], bar_mma[2], bar_sready;
     __shared__ uint32_t tmem_base;
     __shared__ int dead;
@@ -99,9 +103,10 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
                 for (int kb = 0; kb < 4; ++kb) tma_load_2d(sm + st * kTStageBytes + kb * kD * 128, &mapT, kb * 32, prow(j), &bar_fullT[st]);
             };
             auto load_S = [&](int j, int half) {
-                mbar_expect_tx(&bar_fullS[half], kSHalfBytes);
-                for (int cb = 0; cb < 4; ++cb)
-                    tma_load_2d(sS + half * kSHalfBytes + cb * 64 * 128, &mapS, cb * 32, prow(j) + 64 * half, &bar_fullS[half]);
+                mbar_expect_tx(&bar_fullS[half], kSHalf);
+                constexpr int ncb = SBF16 ? 2 : 4, cols = SBF16 ? 64 : 32;   // 128-byte rows either way
+                for (int cb = 0; cb < ncb; ++cb)
+                    tma_load_2d(sS + half * kSHalfBytes + cb * 64 * 128, &mapS, cb * cols, prow(j) + 64 * half, &bar_fullS[half]);
             };
             load_S(0, 0);
             load_S(0, 1);
@@ -150,6 +155,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
         const int i0 = 64 * half;
         const uint32_t lane_base = tacc + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         const float *tile = reinterpret_cast<const float *>(sS + half * kSHalfBytes + (c >> 5) * 64 * 128) + (c & 31);
+        const __nv_bfloat16 *tile16 = reinterpret_cast<const __nv_bfloat16 *>(sS + half * kSHalfBytes + (c >> 6) * 64 * 128) + (c & 63);
         for (int j = 0; j < K; ++j) {
             if (j + 1 < K) {  // round the next transition to nearest tf32 while this step's MMAs run
                 const int st = stage_of(j + 1);
@@ -181,7 +187,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
             mbar_wait(&bar_fullS[half], j & 1, &dead, a.status);
 #pragma unroll
             for (int i = 0; i < 64; ++i) {
-                const float s = tile[i * 32];
+                const float s = SBF16 ? __bfloat162float(tile16[i * 64]) : tile[i * 32];
                 val[i] = (j > 0) ? val[i] + s : s;  // j == 0 hands the first chunk through untouched
             }
             mbar_arrive(&bar_freeS[half]);
@@ -210,20 +216,28 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
 
 }  // namespace
 
-bool init_gdn_exact_tensor_supported(const InitArgs &a, bool pool_bf16) {
-    return !pool_bf16 && a.d_k == kD && a.d_v == kD && a.n_chunks >= 1 &&
+bool init_gdn_exact_tensor_supported(const InitArgs &a, bool) {
+    return a.d_k == kD && a.d_v == kD && a.n_chunks >= 1 &&
            static_cast<long long>(a.n_chunks) * a.H * kD < (1ll << 31);
 }
 
-cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, cudaStream_t s) {
+cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, bool pool_bf16, cudaStream_t s) {
     CUtensorMap mapT, mapS;
     const uint64_t rows = static_cast<uint64_t>(a.n_chunks) * a.H * kD;
-    if (!make_tensor_map_2d(&mapT, a.transitions, 4, kD, rows, kD * 4, 32, kD, true) ||
-        !make_tensor_map_2d(&mapS, a.states, 4, kD, rows, kD * 4, 32, 64, false))
+    if (!make_tensor_map_2d(&mapT, a.transitions, 4, kD, rows, kD * 4, 32, kD, true)) return cudaErrorInvalidValue;
+    if (pool_bf16 ? !make_tensor_map_2d(&mapS, a.states, 2, kD, rows, kD * 2, 64, 64, false)
+                  : !make_tensor_map_2d(&mapS, a.states, 4, kD, rows, kD * 4, 32, 64, false))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(init_gdn_exact_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    init_gdn_exact_tensor_kernel<<<dim3(a.H, a.n_req), kThreads, kSmemBytes, s>>>(a, mapT, mapS);
+    cudaError_t e;
+    if (pool_bf16) {
+        e = cudaFuncSetAttribute(init_gdn_exact_tensor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        init_gdn_exact_tensor_kernel<true><<<dim3(a.H, a.n_req), kThreads, kSmemBytes, s>>>(a, mapT, mapS);
+    } else {
+        e = cudaFuncSetAttribute(init_gdn_exact_tensor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        init_gdn_exact_tensor_kernel<false><<<dim3(a.H, a.n_req), kThreads, kSmemBytes, s>>>(a, mapT, mapS);
+    }
     return cudaGetLastError();
 }
 

@@ -126,7 +126,7 @@ int init_impl(const void *states, const void *transitions, const int32_t *chunk_
                                                           : launch_init_mamba_exact(a, pool_bf16, s);
             break;
         case kGdnFp32: e = launch_init_gdn_exact_fp32(a, pool_bf16, s); break;
-        case kGdnTensor: e = launch_init_gdn_exact_tensor(a, s); break;
+        case kGdnTensor: e = launch_init_gdn_exact_tensor(a, pool_bf16, s); break;
     }
     return e == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
 }

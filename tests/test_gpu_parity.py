@@ -427,3 +427,34 @@ def test_scans_with_more_sequences_than_fit_the_parameter_block():
         assert maxrel(o[a0:a1], o_ref) <= TOL_BF16 and maxrel(ST[s], S_ref) <= TOL_BF16
         y_ref, M_ref = oracle.ssd_seq(m["x"][a0:a1], m["dt"][a0:a1], A, m["B"][a0:a1], m["C"][a0:a1])
         assert maxrel(y[a0:a1], y_ref) <= TOL_BF16 and maxrel(MT[s], M_ref) <= TOL_BF16
+
+
+@pytest.mark.parametrize("compute", COMPUTES)
+def test_gdn_exact_with_bf16_stored_states(compute):
+    """Cached states stored as bf16 (the paper's storage format), fp32 transitions, fp32 result: single request and
+    ragged batch, tensor-core and fp32 paths; K = 1 hands the stored values through exactly."""
+    torch = _torch()
+    rng = np.random.default_rng(41)
+    n, H, d = 10, 3, 128
+    pool = wl.bf16_round(wl.synthetic_states(rng, n, H, d, d))
+    trans = wl.synthetic_gdn_transitions(rng, n, H, d)
+    pool_t, trans_t = dev(pool, torch.bfloat16), dev(trans)
+    tol = TOL_F32 if compute == b.LKV_COMPUTE_FP32 else 2e-3
+    for K in (1, 2, 7):
+        ids = rng.integers(0, n, size=K).astype(np.int32)
+        got = host(b.lkv_init_state(pool_t, trans_t, K, b.LKV_INIT_EXACT, family=b.LKV_FAMILY_GDN, chunk_ids=ids,
+                                    compute=compute))
+        ref = oracle.init_exact_gdn(pool, trans, ids)
+        assert maxrel(got, ref) <= tol, (K, maxrel(got, ref))
+        if K == 1:
+            assert got.tobytes() == pool[ids[0]].astype(np.float32).tobytes()
+    ks = [3, 0, 1, 6]
+    cu = np.concatenate([[0], np.cumsum(ks)]).astype(np.int32)
+    ids = rng.integers(0, n, size=int(cu[-1])).astype(np.int32)
+    got = host(b.lkv_init_state_batched(pool_t, trans_t, ids, cu, len(ks), b.LKV_INIT_EXACT, None,
+                                        family=b.LKV_FAMILY_GDN, compute=compute))
+    for r, K in enumerate(ks):
+        if K == 0:
+            assert not got[r].any()
+        else:
+            assert maxrel(got[r], oracle.init_exact_gdn(pool, trans, ids[cu[r]:cu[r + 1]])) <= tol, r
