@@ -84,9 +84,9 @@ struct SsdArgs {
 // Kernel launchers (one translation unit each); all return a cudaError_t from the launch.
 cudaError_t launch_init_single(const InitArgs &a, bool pool_bf16, cudaStream_t s);
 cudaError_t launch_init_mamba_exact(const InitArgs &a, bool pool_bf16, cudaStream_t s);
-// persistent streaming variant (fp32 pool, head size a multiple of 4096 floats); same results bit for bit
+// persistent streaming variant (head size a multiple of 16 KB of pool values); same results bit for bit
 bool init_mamba_stream_supported(const InitArgs &a, bool pool_bf16);
-cudaError_t launch_init_mamba_exact_stream(const InitArgs &a, cudaStream_t s);
+cudaError_t launch_init_mamba_exact_stream(const InitArgs &a, bool pool_bf16, cudaStream_t s);
 cudaError_t launch_init_gdn_exact_fp32(const InitArgs &a, bool pool_bf16, cudaStream_t s);
 bool init_gdn_exact_tensor_supported(const InitArgs &a, bool pool_bf16);
 cudaError_t launch_init_gdn_exact_tensor(const InitArgs &a, bool pool_bf16, cudaStream_t s);

@@ -122,7 +122,7 @@ int init_impl(const void *states, const void *transitions, const int32_t *chunk_
     switch (which) {
         case kSingle: e = launch_init_single(a, pool_bf16, s); break;
         case kMamba:
-            e = init_mamba_stream_supported(a, pool_bf16) ? launch_init_mamba_exact_stream(a, s)
+            e = init_mamba_stream_supported(a, pool_bf16) ? launch_init_mamba_exact_stream(a, pool_bf16, s)
                                                           : launch_init_mamba_exact(a, pool_bf16, s);
             break;
         case kGdnFp32: e = launch_init_gdn_exact_fp32(a, pool_bf16, s); break;

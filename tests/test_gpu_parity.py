@@ -80,11 +80,12 @@ def _carried(S0, S0_ref, last):
     return maxrel(c, c_ref), share
 
 
+@pytest.mark.parametrize("N", [32, 128])     # 128 x 64: heads are whole 16 KB tiles, the streaming kernel runs
 @pytest.mark.parametrize("pool_bf16", [False, True])
-def test_mamba_exact_synthetic_transitions(pool_bf16):
+def test_mamba_exact_synthetic_transitions(pool_bf16, N):
     torch = _torch()
     rng = np.random.default_rng(3)
-    n, H, N, P = 12, 5, 32, 64
+    n, H, P = 12, 5, 64
     pool = wl.synthetic_states(rng, n, H, N, P)
     if pool_bf16:
         pool = wl.bf16_round(pool)
