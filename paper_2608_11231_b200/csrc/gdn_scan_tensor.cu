@@ -4,26 +4,36 @@
 //
 // Everything is held transposed so that every tensor-core tile has M = d_v = 128 rows (all 128
 // TMEM lanes): lane j owns state column j.  Per block, with cg the running sum of g,
-// gam_t = e^{cg_t}, Gam_ti = e^{cg_t - cg_i}, w_i = e^{cg_C - cg_i} and S the incoming state:
+// gam_t = e^{cg_t}, Gam_ti = e^{cg_t - cg_i}, w_t = e^{cg_C - cg_t} and S the incoming state:
 //   (1) G    = [Q;K] K^T             rows 0..63: q_t.k_i, rows 64..127: k_t.k_i           tcgen05
-//       P_ti = Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)             out warps
+//       Ps_ti = scale Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)      mask warps
 //       M    = (I + A)^{-1}          (UT transform: 16x16 diagonal blocks by substitution in fp32,
 //                                     off-diagonal blocks by tf32 block products)         prep warps
-//   (6) PM   = P M                                                                        tcgen05
-//   (2) D1   = S^T [Q;K]^T           cols 0..63: (S^T q_t)_j, cols 64..127: (S^T k_t)_j    tcgen05
-//       r_t  = beta_t (v_t - gam_t S^T k_t)                                               chain warps
-//   (3) [U^T | (PU)^T] = R^T [M; PM]^T   u = M r solves the block's triangular system     tcgen05
-//       o_t  = scale (gam_t S^T q_t + (P u)_t)                                            out warps
-//   (5) S^T <- gam_C S^T + (U o w)^T K   fp32 state accumulated in TMEM (pre-scaled there) tcgen05
-//       and a bf16 copy of S^T in shared memory is the A operand of (2) for the next block.
-// The prep warps (cumulative decay, the inverse, the bf16 [M; PM] operand) and the mask epilogue of (1)
-// work one block ahead of the chain, so (1), the inverse and (6) are off the block-to-block chain
-// (2) -> r -> (3) -> U o w -> (5) -> state copy.
-// A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
-// Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 out,
-// 12-15 prep (the inverse), 16 TMA loads and the store of the output tile, 17 MMA issue of the chain ((2), (3), (5)),
-// 18 MMA issue of the prep side ((1), (6)), 19 per-block scalars
-// (running up to three blocks ahead).  All waits on mbarriers are bounded.
+//       X_mi = M_mi beta_i           bf16 operand of the block's triangular solve          prep warps
+//  (3a) U^T  = V^T X^T               the part of the solve that does not depend on S       tcgen05
+//  (2K) KS   = S^T K^T               (S^T k_t)_j                                          tcgen05 (A = bf16 S^T in TMEM)
+//       Rk_t = -gam_t KS_t           -> bf16 pairs in place                                chain warps
+//  (3b) U^T += Rk X^T                u = M r, r_t = beta_t (v_t - gam_t S^T k_t): the block's pseudo-values
+//       Uw_t = w_t u_t and u_t       -> two bf16 operands in place                         chain warps
+//   (5) S^T <- gam_C S^T + Uw^T K    fp32 state accumulated in TMEM (pre-scaled there)      tcgen05 (A from TMEM)
+//       S^T -> bf16 pairs in TMEM for (2K)/(2Q) of the next block, pre-scale by its gam_C  chain warps
+//  (2Q) O^T  = S^T Qs^T,  Qs_t = scale gam_t q_t (the Q tile is scaled in place once (1) has read it)
+//   (7) O^T += u^T Ps^T              so that o_t = scale (gam_t S^T q_t + (P u)_t)          tcgen05 (A from TMEM)
+// The block-to-block chain is (2K) -> Rk -> (3b) -> Uw -> (5) -> state copy: three tensor-memory
+// to tensor-memory conversions, no shared memory and no proxy fence on it.  Everything else ((1), the
+// mask epilogue, the inverse, (3a), the Q scaling) runs up to two blocks ahead of the chain; (2Q) and
+// (7) hang off it.  A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
+//
+// Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows; they also turn the
+// finished O^T of the previous block into the output tile while (3b) runs), 8-11 mask epilogue of (1) and Q
+// scaling, 12-15 prep (the inverse), 16 TMA loads of V and the store of the output tile, 17 MMA issue of
+// the chain, 18 TMA loads of Q and K and MMA issue of (1), 19 per-block scalars.  All waits on mbarriers
+// are bounded.
+//
+// The hot loops are kept small on purpose (loops that are not unrolled, rare paths in functions that are not
+// inlined): the twenty warps run seven different programs at once, and with the first, fully unrolled
+// version of this kernel the SMs fetched a third of their instructions from the cache they share with
+// their neighbours, which then ran at 80 % of its request rate and set the pace of the whole kernel.
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -37,44 +47,48 @@ constexpr int kD = 128;   // d_k = d_v
 constexpr int kC = 64;    // tokens per block
 constexpr int kThreads = 640;
 
-// shared-memory map (bytes, after 1024-byte alignment)
-constexpr int kQKStage = 4 * kC * 128;                 // [Q_kb0 | K_kb0 | Q_kb1 | K_kb1], each [64 rows x 128 B]
-constexpr int kOffV = 2 * kQKStage;                    // V tile [64][128] bf16, row-major (single buffer)
-constexpr int kOffSt = kOffV + kC * kD * 2;            // S^T bf16: [St_kb0 | St_kb1], each [128 rows x 128 B]
-constexpr int kOffR = kOffSt + 2 * kD * 128;           // R^T bf16 [128 rows x 128 B]
-constexpr int kOffUw = kOffR;                          // (U o w)^T bf16: written only after (3) has consumed R^T
-constexpr int kOffMPM = kOffR + kD * 128;              // [M; PM] bf16 [128 rows x 128 B], double-buffered; once (3) has read it,
-                                                       // the buffer stages the block's output tile [64 tokens][128] bf16 for the TMA store
-constexpr int kOffP = kOffMPM + 2 * kD * 128;          // P bf16 [64 rows x 128 B] = rows 64..127 of the A operand of (6), whose rows
-                                                       // 0..63 (the end of the [M; PM] buffers) are don't-care: PM lands in TMEM lanes 64..127
+// shared-memory map (bytes, after 1024-byte alignment); operand tiles have 128-byte rows, 128-byte swizzle
+constexpr int kQKStage = 4 * kC * 128;                 // [Q_kb0 | K_kb0 | Q_kb1 | K_kb1], each [64 tokens x 128 B]
+constexpr int kQKStages = 3;                           // (1) and the mask epilogue run two blocks ahead of the chain
+constexpr int kVStage = 2 * kC * 128;                  // [V_jb0 | V_jb1], each [64 tokens x 128 B]; once (3a) has read it, the
+                                                       // stage holds the block's output tile [64 tokens][128] bf16 for the TMA store
+constexpr int kOffV = kQKStages * kQKStage;            // two V stages
+constexpr int kOffX = kOffV + 2 * kVStage;             // X bf16 [64 rows m x 128 B], double-buffered
+constexpr int kOffP = kOffX + 2 * kC * 128;            // Ps bf16 [64 rows t x 128 B], three buffers
 constexpr int kLd = 68;                                // row stride (floats) of the fp32 A and M matrices: rows 4 banks apart
-constexpr int kOffA = kOffP + kC * 128;                // A fp32 [t][i], double-buffered
+constexpr int kOffA = kOffP + 3 * kC * 128;            // A fp32 [t][i], double-buffered
 constexpr int kOffM = kOffA + 2 * kC * kLd * 4;        // M fp32 [t][i]
-constexpr int kOffGb = kOffM + kC * kLd * 4;           // per-block scalars, four buffers (prepared two blocks ahead)
+constexpr int kOffGb = kOffM + kC * kLd * 4;           // per-block scalars, four buffers
 constexpr int kGbFloats = 5 * kC + 4;                  // cg2 = cg log2(e), beta, gam (e^{cg}), w (e^{cg_C - cg}), f (e^{cg_ref - cg}), flag
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kMaxGroupRange = 100.f;                // log2 units: above this the per-group factors could overflow
-constexpr int kSmemUsed = kOffGb + 4 * kGbFloats * 4;   // from the 1024-byte aligned base
-static_assert(kSmemUsed + 1024 <= 227 * 1024, "shared memory budget");
+constexpr int kSmemUsed = kOffGb + 4 * kGbFloats * 4;  // from the 1024-byte aligned base
+constexpr int kSmemBytes = kSmemUsed + 1024;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 // tensor-memory map (columns)
-constexpr uint32_t kTmG = 0;      // 64
-constexpr uint32_t kTmPM = 448;   // 64
-constexpr uint32_t kTmD1 = 64;    // 128: QS | KS
-constexpr uint32_t kTmUP = 192;   // 128: U | PU
-constexpr uint32_t kTmS = 320;    // 128
+constexpr uint32_t kTmS = 0;      // 128: S^T fp32
+constexpr uint32_t kTmSb = 128;   // 64: S^T as bf16 pairs (A operand of (2K), (2Q))
+constexpr uint32_t kTmKS = 192;   // 64: KS fp32; Rk as bf16 pairs in place (tokens 0..31 in columns 0..15, 32..63 in 32..47)
+constexpr uint32_t kTmU = 256;    // 64: U fp32; in place Uw as bf16 pairs (columns 0..15 and 32..47) and u (16..31 and 48..63)
+constexpr uint32_t kTmO = 320;    // 64: O^T
+constexpr uint32_t kTmG = 384;    // 2 x 64: G of the even / odd blocks
 constexpr uint32_t kTmemCols = 512;
 
 struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
-    uint64_t full_qk[2], tiles_free_qk[2], full_v, g_done, pm_done, d1_done, up_done, ds_done, o_free[2];
-    // 128-thread barriers (prep or out warpgroup)
-    uint64_t m_ready[2], o_done[4], inv_done[2], o_staged[2];
-    // 64-thread barriers (the two halves of the out warpgroup)
-    uint64_t a_ready, p_ready, gb_ready[4], mpm_ready[2];
+    uint64_t full_qk[3], tiles_free_qk[3], full_v[2], g_done[2], ks_done, u_done, ds_done, o_mma_done, p_free[3], x_free[2];
+    // 128-thread barriers (prep or mask warpgroup)
+    uint64_t m_ready[2], qs_ready[3];
+    // 64-thread barriers (the two halves of the mask warpgroup)
+    uint64_t a_ready[2], p_ready[3];
+    // 32-thread barriers (the scalar warp)
+    uint64_t gb_ready[4];
     // 256-thread barriers (both chain warpgroups)
-    uint64_t v_free, r_ready, uw_ready, st_ready, chain_done[4];
+    uint64_t rk_ready, uw_ready, st_ready, chain_done[4], o_done[4], o_staged[2];
 };
+constexpr int kBars1 = 19, kBars128 = 5, kBars64 = 5, kBars32 = 4, kBars256 = 13;
+static_assert(sizeof(Bars) == 8 * (kBars1 + kBars128 + kBars64 + kBars32 + kBars256), "barrier table");
 
 __device__ __forceinline__ uint32_t to_tf32(float v) {
     uint32_t r;
@@ -169,6 +183,39 @@ __device__ __forceinline__ void store_row_chunks(unsigned char *tile, int row, i
         *reinterpret_cast<uint4 *>(tile + sw128_offset(row, chunk0 + c8)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
+// 16 fp32 values (as loaded from tensor memory) -> 8 columns of bf16 pairs, the even element in the low half
+__device__ __forceinline__ void pack16(const float (&v)[16], uint32_t (&w)[8]) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(v[2 * e], v[2 * e + 1]);
+}
+// Mask of one group of 16 columns of one row of G, exact form for a block whose decay is too violent for the
+// per-group factors: one exponential per element.  Rare, kept out of the hot loop as a whole (load from tensor
+// memory, mask, store) so that no register array crosses the call.  to_ps: bf16 row of Ps, else fp32 row of A.
+__device__ __noinline__ void mask_group_exact(uint32_t taddr, const float *sc, float cgt, float coef, int i0, int lim, bool to_ps,
+                                              unsigned char *ps, float *arow, int t) {
+    uint32_t rr[16];
+    tmem_ld16(taddr, rr);
+    tmem_ld_wait();
+    float v[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) v[c] = (i0 + c <= lim) ? coef * exp2f(cgt - sc[i0 + c]) * __uint_as_float(rr[c]) : 0.f;
+    if (to_ps) {
+        store_row_chunks(ps, t, i0 >> 3, v);
+    } else {
+#pragma unroll
+        for (int c = 0; c < 16; c += 4) *reinterpret_cast<float4 *>(arow + i0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+    }
+}
+// Rows of a ragged last block go straight to global memory: 16 tokens of one state column per call, read from
+// tensor memory here.
+__device__ __noinline__ void store_o_partial(uint32_t taddr, __nv_bfloat16 *orow, size_t tstride, int n_left) {
+    uint32_t pu[16];
+    tmem_ld16(taddr, pu);
+    tmem_ld_wait();
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        if (c < n_left) orow[c * tstride] = __float2bfloat16_rn(__uint_as_float(pu[c]));
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant__ CUtensorMap mapQ,
@@ -182,19 +229,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, seq = blockIdx.y;
-    {
-        // the launch asks for all the dynamic shared memory the device has left; make sure the aligned map fits
-        uint32_t dyn;
-        asm("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
-        if (static_cast<uint32_t>(sm - smem_raw) + kSmemUsed > dyn) {
-            if (tid == 0 && a.status) atomicExch(a.status, 1);
-            return;
-        }
-    }
     const int hk = h / (a.H_v / a.H_k);
     const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
     const int nblk = (t_end - t_begin + kC - 1) / kC;
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * kD * kD;
+    const bool has_v = a.v != nullptr, has_o = a.o != nullptr;
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
         if (a.S_T && (a.S_T != a.S0 || a.s0_identity))
@@ -204,14 +243,12 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     }
     if (tid == 0) {
         dead = 0;
-        uint64_t *b1 = &bars.full_qk[0];
-        for (int i = 0; i < 12; ++i) mbar_init(b1 + i, 1);
-        uint64_t *b128 = &bars.m_ready[0];
-        for (int i = 0; i < 10; ++i) mbar_init(b128 + i, 128);
-        uint64_t *b64 = &bars.a_ready;
-        for (int i = 0; i < 8; ++i) mbar_init(b64 + i, (i >= 2 && i < 6) ? 32 : 64);   // gb_ready: the scalar warp
-        uint64_t *b256 = &bars.v_free;
-        for (int i = 0; i < 8; ++i) mbar_init(b256 + i, 256);
+        uint64_t *bp = &bars.full_qk[0];
+        for (int i = 0; i < kBars1; ++i) mbar_init(bp++, 1);
+        for (int i = 0; i < kBars128; ++i) mbar_init(bp++, 128);
+        for (int i = 0; i < kBars64; ++i) mbar_init(bp++, 64);
+        for (int i = 0; i < kBars32; ++i) mbar_init(bp++, 32);
+        for (int i = 0; i < kBars256; ++i) mbar_init(bp++, 256);
         mbar_fence_init();
     }
     if (warp == 17) tmem_alloc(&tmem_base, kTmemCols);
@@ -222,51 +259,32 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     float *gb = reinterpret_cast<float *>(sm + kOffGb);
 
     if (warp == 16) {
-        // ======================================================= TMA producer
+        // ======================================================= TMA producer of the V tiles and store of the output tiles
         if (lane == 0) {
-            tma_prefetch_desc(&mapQ);
-            tma_prefetch_desc(&mapK);
-            if (a.v) tma_prefetch_desc(&mapV);
-            if (a.o) tma_prefetch_desc(&mapO);
-            // the output tile of block b (whole blocks only) leaves its staging buffer, the [M; PM] buffer of parity b
-            auto store_o = [&](int b) {
-                mbar_wait(&bars.o_staged[b & 1], (b >> 1) & 1, &dead, a.status);
-                const int t0 = t_begin + b * kC;
-                if (a.o && t0 + kC <= t_end && !dead) {
-                    tma_store_2d(&mapO, sm + kOffMPM + (b & 1) * (kD * 128), h * kD, t0);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
-                mbar_arrive(&bars.o_free[b & 1]);
-            };
-            for (int b = 0; b < nblk; ++b) {
+            if (has_v) tma_prefetch_desc(&mapV);
+            if (has_o) tma_prefetch_desc(&mapO);
+#pragma unroll 1
+            for (int b = 0; b < nblk + 2; ++b) {
                 const int st = b & 1;
                 const int row = t_begin + b * kC;
-                // the two-stage ring cannot hide the DRAM latency of the tile loads: pull the tiles of block b+2 into L2 now
-                if (b + 2 < nblk) {
-                    for (int kb = 0; kb < 2; ++kb) {
-                        tma_prefetch_l2_2d(&mapQ, hk * kD + kb * 64, row + 2 * kC);
-                        tma_prefetch_l2_2d(&mapK, hk * kD + kb * 64, row + 2 * kC);
+                if (has_v && b + 2 < nblk)
+                    for (int kb = 0; kb < 2; ++kb) tma_prefetch_l2_2d(&mapV, h * kD + kb * 64, row + 2 * kC);
+                // the V stage of this parity has held the output tile of block b-2 (whole blocks only) since (3a) of
+                // that block had read it: store the tile, then reuse the stage
+                if (b >= 2) {
+                    mbar_wait(&bars.o_staged[st], ((b - 2) >> 1) & 1, &dead, a.status);
+                    if (has_o && row - kC <= t_end && !dead) {
+                        tma_store_2d(&mapO, sm + kOffV + st * kVStage, h * kD, row - 2 * kC);
+                        tma_store_commit();
+                        tma_store_wait_read();
                     }
-                    if (a.v) tma_prefetch_l2_2d(&mapV, h * kD, row + 2 * kC);
                 }
-                if (b >= 2) mbar_wait(&bars.tiles_free_qk[st], ((b - 2) >> 1) & 1, &dead, a.status);
-                unsigned char *base = sm + st * kQKStage;
-                mbar_expect_tx(&bars.full_qk[st], kQKStage);
-                for (int kb = 0; kb < 2; ++kb) {
-                    tma_load_2d(base + kb * 2 * kC * 128, &mapQ, hk * kD + kb * 64, row, &bars.full_qk[st]);
-                    tma_load_2d(base + kb * 2 * kC * 128 + kC * 128, &mapK, hk * kD + kb * 64, row, &bars.full_qk[st]);
+                if (has_v && b < nblk) {   // without v (read as zeros) nothing is loaded and (3a) is not issued
+                    unsigned char *vb = sm + kOffV + st * kVStage;
+                    mbar_expect_tx(&bars.full_v[st], kVStage);
+                    for (int jb = 0; jb < 2; ++jb) tma_load_2d(vb + jb * kC * 128, &mapV, h * kD + jb * 64, row, &bars.full_v[st]);
                 }
-                if (a.v) {   // without v (read as zeros) nothing is loaded and the chain does not wait for it
-                    if (b >= 1) mbar_wait(&bars.v_free, (b - 1) & 1, &dead, a.status);
-                    mbar_expect_tx(&bars.full_v, kC * kD * 2);
-                    tma_load_2d(sm + kOffV, &mapV, h * kD, row, &bars.full_v);
-                }
-                // the output of block b-2 was staged about one block ago; the inverse of block b needs its buffer only later
-                if (b >= 2) store_o(b - 2);
             }
-            if (nblk >= 2) store_o(nblk - 2);
-            store_o(nblk - 1);
             tma_store_wait_all();
         }
     } else if (warp == 19) {
@@ -285,6 +303,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         };
         float2 gv_next, bv_next;
         fetch_gb(0, gv_next, bv_next);
+#pragma unroll 1
         for (int b = 0; b < nblk; ++b) {
             // the buffer of block b was last read by the chain and the output epilogue of block b-4
             if (b >= 4) {
@@ -295,8 +314,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             float *sc = gb + (b & 3) * kGbFloats;
             const float2 gv = gv_next, bv = bv_next;
             fetch_gb(b + 1, gv_next, bv_next);   // in flight while this block is prepared
-            const float pair = gv.x + gv.y;
-            float run = pair;
+            float run = gv.x + gv.y;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const float up = __shfl_up_sync(0xffffffffu, run, o);
@@ -319,95 +337,127 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_arrive(&bars.gb_ready[b & 3]);
         }
     } else if (warp == 18) {
-        // ======================================================= second MMA issuer: (1) and (6), the prep side
+        // ======================================================= TMA loads of the Q and K tiles (three stages) and MMA issue of (1)
         if (elect_one()) {
-            constexpr uint32_t idG = umma_idesc(kFmtBF16, false, false, 128, 64);    // (1)
-            constexpr uint32_t idPM = umma_idesc(kFmtBF16, false, true, 128, 64);    // (6): B = M read MN-major
-            const uint64_t dP = umma_desc(smem_u32(sm + kOffP - kC * 128), 0, 1024);
-            const uint64_t dMPM0 = umma_desc(smem_u32(sm + kOffMPM), 0, 1024);
-            auto issue_G = [&](int b) {
-                const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
-#pragma unroll
+            constexpr uint32_t idG = umma_idesc(kFmtBF16, false, false, 128, 64);
+            tma_prefetch_desc(&mapQ);
+            tma_prefetch_desc(&mapK);
+#pragma unroll 1
+            for (int b = 0; b < nblk; ++b) {
+                const int s3 = b % kQKStages;
+                const int row = t_begin + b * kC;
+                unsigned char *base = sm + s3 * kQKStage;
+                // the tiles of block b go into the stage that (5) of block b-3 has released: two blocks before the
+                // chain needs them.  The ring cannot hide the DRAM latency: the tiles of block b+3 are pulled into L2 now.
+#pragma unroll 1
+                for (int kb = 0; kb < 2; ++kb) {
+                    if (b + kQKStages < nblk) {
+                        tma_prefetch_l2_2d(&mapQ, hk * kD + kb * 64, row + kQKStages * kC);
+                        tma_prefetch_l2_2d(&mapK, hk * kD + kb * 64, row + kQKStages * kC);
+                    }
+                }
+                if (b >= kQKStages) mbar_wait(&bars.tiles_free_qk[s3], ((b - kQKStages) / kQKStages) & 1, &dead, a.status);
+                mbar_expect_tx(&bars.full_qk[s3], kQKStage);
+#pragma unroll 1
+                for (int kb = 0; kb < 2; ++kb) {
+                    tma_load_2d(base + kb * 2 * kC * 128, &mapQ, hk * kD + kb * 64, row, &bars.full_qk[s3]);
+                    tma_load_2d(base + kb * 2 * kC * 128 + kC * 128, &mapK, hk * kD + kb * 64, row, &bars.full_qk[s3]);
+                }
+                // (1) of block b: the mask epilogue of block b-2 has drained these G columns
+                if (b >= 2) {
+                    mbar_wait(&bars.a_ready[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+                    mbar_wait(&bars.p_ready[(b - 2) % 3], ((b - 2) / 3) & 1, &dead, a.status);
+                }
+                mbar_wait(&bars.full_qk[s3], (b / kQKStages) & 1, &dead, a.status);
+                tc_fence_after_sync();
+                const uint64_t dQK = umma_desc(smem_u32(base), 0, 1024);
+#pragma unroll 1
                 for (int k = 0; k < 8; ++k) {
                     const uint64_t off = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
-                    umma_bf16(tm + kTmG, dQK + off, dQK + off + ((kC * 128) >> 4), idG, k > 0);
+                    umma_bf16(tm + kTmG + 64 * (b & 1), dQK + off, dQK + off + ((kC * 128) >> 4), idG, k > 0);
                 }
-                umma_commit(&bars.g_done);
-            };
-            mbar_wait(&bars.full_qk[0], 0, &dead, a.status);
-            tc_fence_after_sync();
-            issue_G(0);
-            for (int b = 0; b < nblk; ++b) {
-                const uint32_t par = b & 1;
-                // (1) of the next block as soon as the mask epilogue of this one has drained the G columns
-                if (b + 1 < nblk) {
-                    mbar_wait(&bars.a_ready, par, &dead, a.status);
-                    mbar_wait(&bars.p_ready, par, &dead, a.status);
-                    mbar_wait(&bars.full_qk[(b + 1) & 1], ((b + 1) >> 1) & 1, &dead, a.status);
-                    tc_fence_after_sync();
-                    issue_G(b + 1);
-                }
-                // (6) of this block as soon as its inverse is there: PM = P M, A = P (K = i), B = M rows of [M; PM] read MN-major
-                mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
-                mbar_wait(&bars.p_ready, par, &dead, a.status);
-                // the accumulator of (6) must have been read for block b-1 (its PM rows are in the operand)
-                if (b >= 1) mbar_wait(&bars.mpm_ready[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
-                tc_fence_after_sync();
-                const uint64_t dM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
-#pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmPM, dP + 2 * k, dM + ((k * 16 * 128) >> 4), idPM, k > 0);
-                umma_commit(&bars.pm_done);
+                umma_commit(&bars.g_done[b & 1]);
             }
         }
     } else if (warp == 17) {
-        // ======================================================= first MMA issuer: (2), (3), (5), the block-to-block chain
+        // ======================================================= first MMA issuer: (2K), (3a), (3b), (2Q), (5), (7)
         if (elect_one()) {
-            constexpr uint32_t idD1 = umma_idesc(kFmtBF16, false, false, 128, 128);  // (2), (3)
-            constexpr uint32_t idDS = umma_idesc(kFmtBF16, false, true, 128, 128);   // (5): B = K tile read MN-major
-            const uint64_t dSt = umma_desc(smem_u32(sm + kOffSt), 0, 1024);
-            const uint64_t dR = umma_desc(smem_u32(sm + kOffR), 0, 1024);
-            const uint64_t dUw = umma_desc(smem_u32(sm + kOffUw), 0, 1024);
-            const uint64_t dMPM0 = umma_desc(smem_u32(sm + kOffMPM), 0, 1024);
+            constexpr uint32_t idN64 = umma_idesc(kFmtBF16, false, false, 128, 64);    // (2K), (2Q), (3b), (7)
+            constexpr uint32_t id3a = umma_idesc(kFmtBF16, true, false, 128, 64);      // A = V tile read MN-major
+            constexpr uint32_t id5 = umma_idesc(kFmtBF16, false, true, 128, 128);      // B = K tile read MN-major
+#pragma unroll 1
             for (int b = 0; b < nblk; ++b) {
                 const uint32_t par = b & 1;
-                const uint64_t dQK = umma_desc(smem_u32(sm + (b & 1) * kQKStage), 0, 1024);
-                // (2) needs the bf16 state copy of block b, the D1 / UP accumulators drained, and the Q / K tiles
+                const uint32_t qk = smem_u32(sm + (b % kQKStages) * kQKStage);
+                const uint64_t dQ = umma_desc(qk, 0, 1024), dK = umma_desc(qk + kC * 128, 0, 1024);
+                const uint64_t dX = umma_desc(smem_u32(sm + kOffX + (b & 1) * (kC * 128)), 0, 1024);
+                // (2K) needs the bf16 state of block b and the K tile
                 mbar_wait(&bars.st_ready, par, &dead, a.status);
-                if (b > 0) mbar_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1, &dead, a.status);
-                mbar_wait(&bars.full_qk[b & 1], (b >> 1) & 1, &dead, a.status);
+                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
                 tc_fence_after_sync();
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const uint64_t offA = ((k >> 2) * (kD * 128) + (k & 3) * 32) >> 4;
-                    const uint64_t offB = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
-                    umma_bf16(tm + kTmD1, dSt + offA, dQK + offB, idD1, k > 0);
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16_ts(tm + kTmKS, tm + kTmSb + 8 * k, dK + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
+                umma_commit(&bars.ks_done);
+                // (3a) U = V^T X^T: needs the inverse of the block and the V tile (the U columns were read by (5) and (7)
+                // of the previous block, issued before)
+                mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+                if (has_v) {
+                    mbar_wait(&bars.full_v[b & 1], (b >> 1) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+                    const uint64_t dV = umma_desc(smem_u32(sm + kOffV + (b & 1) * kVStage), kC * 128, 1024);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmU, dV + ((k * 16 * 128) >> 4), dX + 2 * k, id3a, k > 0);
                 }
-                umma_commit(&bars.d1_done);
-                // (3) [U | PU] = R^T [M; PM]^T
-                mbar_wait(&bars.mpm_ready[b & 1], (b >> 1) & 1, &dead, a.status);
-                mbar_wait(&bars.r_ready, par, &dead, a.status);
+                // (3b) U += Rk X^T
+                mbar_wait(&bars.rk_ready, par, &dead, a.status);
                 tc_fence_after_sync();
-                const uint64_t dMPM = dMPM0 + ((b & 1) * ((kD * 128) >> 4));
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmUP, dR + 2 * k, dMPM + 2 * k, idD1, k > 0);
-                umma_commit(&bars.up_done);
+                for (int k = 0; k < 4; ++k)
+                    umma_bf16_ts(tm + kTmU, tm + kTmKS + 32 * (k >> 1) + 8 * (k & 1), dX + 2 * k, idN64, has_v || k > 0);
+                umma_commit(&bars.u_done);
+                umma_commit(&bars.x_free[b & 1]);
+                // (2Q) O = S^T Qs^T behind (3b): the chain warps drain the O columns of the previous block while (3b)
+                // runs, before they turn to U, so this wait never outlasts the next one
+                if (has_o) {
+                    if (b > 0) mbar_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1, &dead, a.status);
+                    mbar_wait(&bars.qs_ready[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16_ts(tm + kTmO, tm + kTmSb + 8 * k, dQ + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
+                }
                 // (5) accumulates onto the pre-scaled state; B = K tile read MN-major (rows = tokens)
                 mbar_wait(&bars.uw_ready, par, &dead, a.status);
                 tc_fence_after_sync();
-                const uint64_t dKmn = umma_desc(smem_u32(sm + (b & 1) * kQKStage + kC * 128), 2 * kC * 128, 1024);
+                const uint64_t dKmn = umma_desc(qk + kC * 128, 2 * kC * 128, 1024);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16(tm + kTmS, dUw + 2 * k, dKmn + ((k * 16 * 128) >> 4), idDS, true);
+                for (int k = 0; k < 4; ++k)
+                    umma_bf16_ts(tm + kTmS, tm + kTmU + 32 * (k >> 1) + 8 * (k & 1), dKmn + ((k * 16 * 128) >> 4), id5, true);
                 umma_commit(&bars.ds_done);
-                umma_commit(&bars.tiles_free_qk[b & 1]);
+                umma_commit(&bars.tiles_free_qk[b % kQKStages]);
+                // (7) O += u^T Ps^T
+                if (has_o) {
+                    mbar_wait(&bars.p_ready[b % 3], (b / 3) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+                    const uint64_t dP = umma_desc(smem_u32(sm + kOffP + (b % 3) * (kC * 128)), 0, 1024);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16_ts(tm + kTmO, tm + kTmU + 32 * (k >> 1) + 16 + 8 * (k & 1), dP + 2 * k, idN64, true);
+                    umma_commit(&bars.p_free[b % 3]);
+                }
+                umma_commit(&bars.o_mma_done);
             }
         }
     } else if (warp >= 12) {
-        // ======================================================= prep warpgroup: the inverse, ahead of the chain
+        // ======================================================= prep warpgroup: the inverse and its operand, ahead of the chain
         const int x = tid - 384;                 // 0..127
         float *Mf = reinterpret_cast<float *>(sm + kOffM);
+#pragma unroll 1
         for (int b = 0; b < nblk; ++b) {
-            // ---- P and A come from the out warpgroup (epilogue of (1))
-            mbar_wait(&bars.a_ready, b & 1, &dead, a.status);
+            const float *sc = gb + (b & 3) * kGbFloats;
+            // ---- A comes from the mask warpgroup (epilogue of (1))
+            mbar_wait(&bars.a_ready[b & 1], (b >> 1) & 1, &dead, a.status);
             named_bar_sync(1, 128);   // every thread is done with the fp32 M of the previous block
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
             // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k by forward
@@ -449,219 +499,149 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 if (wq < 2) inv_offdiag<1, 3>(Af, Mf, 0, wq, gid, tig);
                 named_bar_sync(1, 128);
             }
-            // ---- M as bf16 operand rows 0..63 of [M; PM] (zeros above the block diagonal)
-            // the [M; PM] buffer of this parity was read by (3) of block b-2 and then staged that block's output tile
-            if (b >= 2) mbar_wait(&bars.o_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-            unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
+            // ---- X = M diag(beta) as bf16 operand (zeros above the block diagonal); the buffer of this parity was
+            // read by (3b) of block b-2
+            if (b >= 2) mbar_wait(&bars.x_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+            unsigned char *xb = sm + kOffX + (b & 1) * (kC * 128);
             {
-                // thread = (row t, half of the columns)
-                const int t = x & 63, q0 = 2 * (x >> 6);
-#pragma unroll
+                // thread = (row m, half of the columns)
+                const int m = x & 63, q0 = 2 * (x >> 6);
+#pragma unroll 1
                 for (int q = q0; q < q0 + 2; ++q) {
                     float v[16];
+                    const bool live = q <= (m >> 4);
 #pragma unroll
                     for (int c = 0; c < 16; c += 4) {
                         const int i = 16 * q + c;
-                        const float4 mv = (i >> 4) <= (t >> 4) ? *reinterpret_cast<const float4 *>(Mf + t * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        v[c] = mv.x; v[c + 1] = mv.y; v[c + 2] = mv.z; v[c + 3] = mv.w;
+                        const float4 mv = live ? *reinterpret_cast<const float4 *>(Mf + m * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float4 be = *reinterpret_cast<const float4 *>(sc + kC + i);
+                        v[c] = mv.x * be.x; v[c + 1] = mv.y * be.y; v[c + 2] = mv.z * be.z; v[c + 3] = mv.w * be.w;
                     }
-                    store_row_chunks(mpm, t, 2 * q, v);
+                    store_row_chunks(xb, m, 2 * q, v);
                 }
             }
             fence_async_smem();
             mbar_arrive(&bars.m_ready[b & 1]);
-            mbar_arrive(&bars.inv_done[b & 1]);
         }
     } else if (warp >= 8) {
-        // ======================================================= out warpgroup: o_t[j] = scale (gam_t (S^T q_t)_j + (P u)_t[j]); lane = j
-        const int j = tid - 256;
+        // ======================================================= mask warpgroup: epilogue of (1) and Q scaling, as far ahead of the
+        // chain as the buffers allow
+        const int x = tid - 256;   // TMEM lane: 0..63 rows of Q K^T (-> Ps), 64..127 rows of K K^T (-> A)
+        const int t = x & 63;
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
-        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
-        const int x = j;   // TMEM lane: 0..63 rows of Q K^T (-> P), 64..127 rows of K K^T (-> A)
-        // epilogue of (1) for block b: P (bf16 operand of (6)) and A (fp32, input of the inverse)
-        // PM rows of block b (lanes 64..127 of the (6) accumulator) -> rows 64..127 of [M; PM]; warps 10 and 11 only,
-        // so that the P rows of the next block (warps 8 and 9) are worked on at the same time
-        auto pm_rows = [&](int b) {
-            mbar_wait(&bars.pm_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            unsigned char *mpm = sm + kOffMPM + (b & 1) * (kD * 128);
-#pragma unroll 1
-            for (int q = 0; q < 4; ++q) {
-                uint32_t rr[16];
-                tmem_ld16(lane_base + kTmPM + 16 * q, rr);
-                tmem_ld_wait();
-                float v[16];
-#pragma unroll
-                for (int c = 0; c < 16; ++c) v[c] = __uint_as_float(rr[c]);
-                store_row_chunks(mpm, x, 2 * q, v);
-            }
-            fence_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&bars.mpm_ready[b & 1]);
-        };
-        auto g_epilogue = [&](int b) {
-            const float *sc = gb + (b & 3) * kGbFloats;
-            mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
-            float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
-            bool pm_pending = x >= kC && b >= 1;
-            if (x < kC) {
-                // the P buffer is free once (6) of block b-1 has read it
-                if (b >= 1) mbar_wait(&bars.pm_done, (b - 1) & 1, &dead, a.status);
-            } else {
-                // the A buffer of this parity is free once block b-2 has been inverted
-                if (b >= 2) mbar_wait(&bars.inv_done[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                // the result of (6) of block b-1 is on the chain's critical path: take it first if it is there already
-                if (pm_pending && __all_sync(0xffffffffu, mbar_test_wait(&bars.pm_done, (b - 1) & 1))) {
-                    pm_rows(b - 1);
-                    pm_pending = false;
-                }
-            }
-            mbar_wait(&bars.g_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            {
-                // Gam_ti = 2^{cg2_t - cg2_ref} * f_i with ref the first column of i's group of 16: one exponential
-                // per group (both factors' product is <= 1 where i <= t); violent decay takes the per-element path
-                const int t = x & 63;
-                const float cgt = sc[t];
-                const float coef = (x < kC) ? 1.f : sc[kC + t];     // rows of P: 1, rows of A: beta_t
-                const int lim = (x < kC) ? t : t - 1;               // P keeps the diagonal, A is strictly lower
-                const bool fast = sc[5 * kC] + sc[5 * kC + 1] == 0.f;
-                const int row_hi = (t & 32) + 31;   // last row (token) of this warp
-#pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    const int i0 = 16 * q;
-                    if (i0 > row_hi) break;   // above the diagonal for every row of this warp: zeroed once, never written
-                    uint32_t rr[16];
-                    tmem_ld16(lane_base + kTmG + 16 * q, rr);
-                    tmem_ld_wait();
-                    float v[16];
-                    if (fast) {
-                        float aa;
-                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(cgt - sc[i0], 0.f)));
-                        aa *= coef;
-                        if (i0 + 15 <= row_hi - 32) {
-                            // below the diagonal for every row of this warp: no masking
-#pragma unroll
-                            for (int c = 0; c < 16; c += 4) {
-                                const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                                v[c] = __uint_as_float(rr[c]) * aa * f.x;
-                                v[c + 1] = __uint_as_float(rr[c + 1]) * aa * f.y;
-                                v[c + 2] = __uint_as_float(rr[c + 2]) * aa * f.z;
-                                v[c + 3] = __uint_as_float(rr[c + 3]) * aa * f.w;
-                            }
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < 16; c += 4) {
-                                const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                                v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
-                                v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
-                                v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
-                                v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            v[c] = (i0 + c <= lim) ? coef * exp2f(cgt - sc[i0 + c]) * __uint_as_float(rr[c]) : 0.f;
-                    }
-                    if (x < kC) {
-                        store_row_chunks(sm + kOffP, t, 2 * q, v);
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 16; c += 4)
-                            *reinterpret_cast<float4 *>(Af + t * kLd + 16 * q + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                    }
-                }
-            }
-            tc_fence_before_sync();
-            if (x < kC) {
-                fence_async_smem();
-                mbar_arrive(&bars.p_ready);
-            } else {
-                mbar_arrive(&bars.a_ready);
-            }
-            if (pm_pending) pm_rows(b - 1);
-        };
+        const int row_hi = (t & 32) + 31;   // last row (token) of this warp
         if ((x & 32) == 0) {
-            // columns 32..63 of rows 0..31 lie above the diagonal in P and in both A buffers: zero them once
-            const int t = x & 63;
+            // columns 32..63 of rows 0..31 lie above the diagonal in all Ps and A buffers: zero them once
             float z[16];
 #pragma unroll
             for (int c = 0; c < 16; ++c) z[c] = 0.f;
-            for (int q = 2; q < 4; ++q) {
+#pragma unroll 1
+            for (int i = 0; i < 6; ++i) {
+                const int q = 2 + (i & 1), bufi = i >> 1;
                 if (x < kC) {
-                    store_row_chunks(sm + kOffP, t, 2 * q, z);
-                } else {
-                    for (int bufi = 0; bufi < 2; ++bufi)
-                        for (int c = 0; c < 16; c += 4)
-                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sm + kOffA) + bufi * (kC * kLd) + t * kLd + 16 * q + c) =
-                                make_float4(0.f, 0.f, 0.f, 0.f);
+                    store_row_chunks(sm + kOffP + bufi * (kC * 128), t, 2 * q, z);
+                } else if (bufi < 2) {
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4)
+                        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sm + kOffA) + bufi * (kC * kLd) + t * kLd + 16 * q + c) =
+                            make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
         }
-        g_epilogue(0);
+#pragma unroll 1
         for (int b = 0; b < nblk; ++b) {
-            if (b + 1 < nblk) g_epilogue(b + 1);   // while the chain works on block b
-            else if (x >= kC) pm_rows(b);
             const float *sc = gb + (b & 3) * kGbFloats;
-            mbar_wait(&bars.d1_done, b & 1, &dead, a.status);
-            mbar_wait(&bars.up_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            const int t0 = t_begin + b * kC;
-            const int n = min(kC, t_end - t0);
-            if (!a.o) {
-                // no outputs wanted (final state only): nothing to drain
-            } else if (n == kC) {
-                // whole block: stage the tile [token][j] in the [M; PM] buffer of this block, which (3) has finished
-                // reading (up_done); the store warp writes it out with TMA
-                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffMPM + (b & 1) * (kD * 128)) + j;
-#pragma unroll 1
-                for (int q = 0; q < 8; ++q) {
-                    uint32_t qs[8], pu[8];
-                    tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
-                    tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
-                    tmem_ld_wait();
-                    const float4 g0 = *reinterpret_cast<const float4 *>(sc + 2 * kC + 8 * q);
-                    const float4 g1 = *reinterpret_cast<const float4 *>(sc + 2 * kC + 8 * q + 4);
-                    const float gm[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        os[(8 * q + c) * kD] = __float2bfloat16_rn(a.scale * fmaf(gm[c], __uint_as_float(qs[c]), __uint_as_float(pu[c])));
-                }
-                fence_async_smem();
+            mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
+            float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
+            unsigned char *ps = sm + kOffP + (b % 3) * (kC * 128);
+            if (x < kC) {
+                // the Ps buffer is free once (7) of block b-3 has read it
+                if (b >= 3 && has_o) mbar_wait(&bars.p_free[b % 3], ((b - 3) / 3) & 1, &dead, a.status);
             } else {
-                __nv_bfloat16 *orow = o + (static_cast<size_t>(t0) * a.H_v + h) * kD + j;
+                // the A buffer of this parity is free once block b-2 has been inverted
+                if (b >= 2) mbar_wait(&bars.m_ready[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+            }
+            mbar_wait(&bars.g_done[b & 1], (b >> 1) & 1, &dead, a.status);
+            tc_fence_after_sync();
+            if (x >= kC || has_o) {
+                // Gam_ti = 2^{cg2_t - cg2_ref} * f_i with ref the first column of i's group of 16: one exponential
+                // per group (both factors' product is <= 1 where i <= t); violent decay takes the per-element path
+                const float cgt = sc[t];
+                const float coef = (x < kC) ? a.scale : sc[kC + t];     // rows of Ps: the output scale, rows of A: beta_t
+                const int lim = (x < kC) ? t : t - 1;                   // P keeps the diagonal, A is strictly lower
+                const bool fast = sc[5 * kC] + sc[5 * kC + 1] == 0.f;
+                const uint32_t tmg = lane_base + kTmG + 64 * (b & 1);
+                // column groups above the diagonal for every row of this warp are never touched
 #pragma unroll 1
-                for (int q = 0; q < 8; ++q) {
-                    uint32_t qs[8], pu[8];
-                    tmem_ld8(lane_base + kTmD1 + 8 * q, qs);
-                    tmem_ld8(lane_base + kTmUP + kC + 8 * q, pu);
+                for (int q = 0; 16 * q <= row_hi; ++q) {
+                    const int i0 = 16 * q;
+                    if (!fast) {
+                        mask_group_exact(tmg + i0, sc, cgt, coef, i0, lim, x < kC, ps, Af + t * kLd, t);
+                        continue;
+                    }
+                    uint32_t rr[16];
+                    tmem_ld16(tmg + i0, rr);
                     tmem_ld_wait();
+                    float v[16];
+                    float aa;
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(cgt - sc[i0], 0.f)));
+                    aa *= coef;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const int t = 8 * q + c;
-                        const float val = a.scale * fmaf(sc[2 * kC + t], __uint_as_float(qs[c]), __uint_as_float(pu[c]));
-                        if (t < n) orow[t * tstride] = __float2bfloat16_rn(val);
+                    for (int c = 0; c < 16; c += 4) {
+                        const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                        v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                        v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                        v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                        v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                    }
+                    if (x < kC) {
+                        store_row_chunks(ps, t, 2 * q, v);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; c += 4)
+                            *reinterpret_cast<float4 *>(Af + t * kLd + i0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
                     }
                 }
             }
             tc_fence_before_sync();
-            mbar_arrive(&bars.o_done[b & 3]);
-            mbar_arrive(&bars.o_staged[b & 1]);
+            if (x < kC) {
+                fence_async_smem();
+                mbar_arrive(&bars.p_ready[b % 3]);
+            } else {
+                mbar_arrive(&bars.a_ready[b & 1]);
+            }
+            // Q tile of block b scaled in place by scale gam_t now that (1) has read it: thread = (token, 64-column half)
+            if (has_o) {
+                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);   // this thread reads what the TMA wrote
+                unsigned char *qt = sm + (b % kQKStages) * kQKStage + (x >> 6) * (2 * kC * 128) + t * 128;
+                const __nv_bfloat162 f2 = __float2bfloat162_rn(a.scale * sc[2 * kC + t]);
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    uint4 *p = reinterpret_cast<uint4 *>(qt + ((c ^ (t & 7)) << 4));
+                    uint4 v = *p;
+                    __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) e[i] = __hmul2(e[i], f2);
+                    *p = v;
+                }
+                fence_async_smem();
+                mbar_arrive(&bars.qs_ready[b % kQKStages]);
+            }
         }
     } else {
         // ======================================================= chain warpgroups: lane = state column j, `half` = token / row half
         const int j = tid & 127, half = warp >> 2;
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        // initial state: S0[m][j], m = 64*half..+63 -> TMEM (fp32, pre-scaled by gam_C of block 0) and bf16 copy
+        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
+        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
+        // initial state: S0[m][j], m = 64*half..+63 -> TMEM (fp32, pre-scaled by gam_C of block 0) and bf16 pairs
         mbar_wait(&bars.gb_ready[0], 0, &dead, a.status);
         {
             const float gamC = gb[2 * kC + kC - 1];
 #pragma unroll 1
             for (int q = 0; q < 4; ++q) {
                 float v[16];
-                uint32_t rr[16];
+                uint32_t rr[16], w[8];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const int m = 64 * half + 16 * q + c;
@@ -669,105 +649,151 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     rr[c] = __float_as_uint(v[c] * gamC);
                 }
                 tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);
-                store_row_chunks(sm + kOffSt + half * (kD * 128), j, 2 * q, v);
+                pack16(v, w);
+                tmem_st8(lane_base + kTmSb + 32 * half + 8 * q, w);
             }
             tmem_st_wait();
-            fence_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&bars.st_ready);
         }
-        for (int b = 0; b < nblk; ++b) {
+        // outputs of block b: O^T (complete once (7) has run) -> bf16 tile, tokens 32*half..+31
+        auto o_epilogue = [&](int b) {
+            mbar_wait(&bars.o_mma_done, b & 1, &dead, a.status);
+            tc_fence_after_sync();
+            const int t0 = t_begin + b * kC;
+            const int n = min(kC, t_end - t0);
+            if (has_o && (n == kC || !dead)) {
+                // whole block: stage the tile [token][j] in the V stage of this block, which (3a) has finished
+                // reading; the store warp writes it out with TMA
+                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffV + (b & 1) * kVStage) + (32 * half) * kD + j;
+#pragma unroll 1
+                for (int q = 0; q < 2; ++q) {
+                    const uint32_t taddr = lane_base + kTmO + 32 * half + 16 * q;
+                    if (n != kC) {
+                        store_o_partial(taddr, o + (static_cast<size_t>(t0 + 32 * half + 16 * q) * a.H_v + h) * kD + j, tstride, n - 32 * half - 16 * q);
+                        continue;
+                    }
+                    uint32_t pu[16];
+                    tmem_ld16(taddr, pu);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) os[(16 * q + c) * kD] = __float2bfloat16_rn(__uint_as_float(pu[c]));
+                }
+                fence_async_smem();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars.o_done[b & 3]);
+            mbar_arrive(&bars.o_staged[b & 1]);
+        };
+#pragma unroll 1
+        for (int b = 0; b <= nblk; ++b) {
+            if (b == nblk) {   // the outputs of the last block
+                o_epilogue(b - 1);
+                break;
+            }
             const uint32_t par = b & 1;
             const float *sc = gb + (b & 3) * kGbFloats;
-            const __nv_bfloat16 *vt = reinterpret_cast<const __nv_bfloat16 *>(sm + kOffV);
             if (b > 0) mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
-            const bool has_v = a.v != nullptr;
-            if (has_v) mbar_wait(&bars.full_v, par, &dead, a.status);
-            mbar_wait(&bars.d1_done, par, &dead, a.status);
+            mbar_wait(&bars.ks_done, par, &dead, a.status);
             tc_fence_after_sync();
-            // r_t = beta_t (v_t[j] - gam_t (S^T k_t)_j), t = 32*half..+31 -> R^T row j
-#pragma unroll 1
-            for (int q = 0; q < 2; ++q) {
-                uint32_t rr[16];
-                tmem_ld16(lane_base + kTmD1 + kC + 32 * half + 16 * q, rr);
+            // Rk_t[j] = -gam_t (S^T k_t)_j, t = 32*half..+31 -> bf16 pairs over the first half of this thread's own columns
+            {
+                uint32_t rr[2][16], w[2][8];
+                tmem_ld16(lane_base + kTmKS + 32 * half, rr[0]);
+                tmem_ld16(lane_base + kTmKS + 32 * half + 16, rr[1]);
                 tmem_ld_wait();
-                float v[16];
 #pragma unroll
-                for (int c = 0; c < 16; c += 4) {
-                    const int t = 32 * half + 16 * q + c;
-                    const float4 be = *reinterpret_cast<const float4 *>(sc + kC + t);
-                    const float4 ga = *reinterpret_cast<const float4 *>(sc + 2 * kC + t);
-                    const float v0 = has_v ? __bfloat162float(vt[t * kD + j]) : 0.f;
-                    const float v1 = has_v ? __bfloat162float(vt[(t + 1) * kD + j]) : 0.f;
-                    const float v2 = has_v ? __bfloat162float(vt[(t + 2) * kD + j]) : 0.f;
-                    const float v3 = has_v ? __bfloat162float(vt[(t + 3) * kD + j]) : 0.f;
-                    v[c] = be.x * (v0 - ga.x * __uint_as_float(rr[c]));
-                    v[c + 1] = be.y * (v1 - ga.y * __uint_as_float(rr[c + 1]));
-                    v[c + 2] = be.z * (v2 - ga.z * __uint_as_float(rr[c + 2]));
-                    v[c + 3] = be.w * (v3 - ga.w * __uint_as_float(rr[c + 3]));
+                for (int q = 0; q < 2; ++q) {
+                    float v[16];
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4) {
+                        const float4 ga = *reinterpret_cast<const float4 *>(sc + 2 * kC + 32 * half + 16 * q + c);
+                        v[c] = -ga.x * __uint_as_float(rr[q][c]);
+                        v[c + 1] = -ga.y * __uint_as_float(rr[q][c + 1]);
+                        v[c + 2] = -ga.z * __uint_as_float(rr[q][c + 2]);
+                        v[c + 3] = -ga.w * __uint_as_float(rr[q][c + 3]);
+                    }
+                    pack16(v, w[q]);
                 }
-                store_row_chunks(sm + kOffR, j, 4 * half + 2 * q, v);
+                tmem_st8(lane_base + kTmKS + 32 * half, w[0]);
+                tmem_st8(lane_base + kTmKS + 32 * half + 8, w[1]);
             }
-            mbar_arrive(&bars.v_free);
-            fence_async_smem();
+            tmem_st_wait();
             tc_fence_before_sync();
-            mbar_arrive(&bars.r_ready);
-            // (U o w)^T row j, i = 32*half..+31
-            mbar_wait(&bars.up_done, par, &dead, a.status);
+            mbar_arrive(&bars.rk_ready);
+            // while (3b) runs: the outputs of the previous block
+            if (b > 0) o_epilogue(b - 1);
+            // u_t[j], tokens 32*half..+31 -> Uw = w o u as bf16 pairs over the first 16 of this thread's own 32 columns, u over the rest
+            mbar_wait(&bars.u_done, par, &dead, a.status);
             tc_fence_after_sync();
-#pragma unroll 1
-            for (int q = 0; q < 2; ++q) {
-                uint32_t rr[16];
-                tmem_ld16(lane_base + kTmUP + 32 * half + 16 * q, rr);
+            {
+                uint32_t rr[2][16], w[2][8], u[2][8];
+                tmem_ld16(lane_base + kTmU + 32 * half, rr[0]);
+                tmem_ld16(lane_base + kTmU + 32 * half + 16, rr[1]);
                 tmem_ld_wait();
-                float v[16];
 #pragma unroll
-                for (int c = 0; c < 16; c += 4) {
-                    const float4 w4 = *reinterpret_cast<const float4 *>(sc + 3 * kC + 32 * half + 16 * q + c);
-                    v[c] = __uint_as_float(rr[c]) * w4.x;
-                    v[c + 1] = __uint_as_float(rr[c + 1]) * w4.y;
-                    v[c + 2] = __uint_as_float(rr[c + 2]) * w4.z;
-                    v[c + 3] = __uint_as_float(rr[c + 3]) * w4.w;
+                for (int q = 0; q < 2; ++q) {
+                    float v[16];
+#pragma unroll
+                    for (int c = 0; c < 16; c += 4) {
+                        const float4 w4 = *reinterpret_cast<const float4 *>(sc + 3 * kC + 32 * half + 16 * q + c);
+                        v[c] = w4.x * __uint_as_float(rr[q][c]);
+                        v[c + 1] = w4.y * __uint_as_float(rr[q][c + 1]);
+                        v[c + 2] = w4.z * __uint_as_float(rr[q][c + 2]);
+                        v[c + 3] = w4.w * __uint_as_float(rr[q][c + 3]);
+                    }
+                    pack16(v, w[q]);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) u[q][e] = pack_bf16(__uint_as_float(rr[q][2 * e]), __uint_as_float(rr[q][2 * e + 1]));
                 }
-                store_row_chunks(sm + kOffUw, j, 4 * half + 2 * q, v);
+                tmem_st8(lane_base + kTmU + 32 * half, w[0]);
+                tmem_st8(lane_base + kTmU + 32 * half + 8, w[1]);
+                tmem_st8(lane_base + kTmU + 32 * half + 16, u[0]);
+                tmem_st8(lane_base + kTmU + 32 * half + 24, u[1]);
             }
-            fence_async_smem();
+            tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(&bars.uw_ready);
-            // new state rows m = 64*half..+63: bf16 copy for the next block and pre-scale by its gam_C, or S_T at the end
-            mbar_wait(&bars.ds_done, par, &dead, a.status);
-            tc_fence_after_sync();
+            // new state rows m = 64*half..+63: bf16 pairs for the next block and pre-scale by its gam_C, or S_T at the end
             const bool last = b + 1 == nblk;
             float gamN = 1.f;
             if (!last) {
                 mbar_wait(&bars.gb_ready[(b + 1) & 3], ((b + 1) >> 2) & 1, &dead, a.status);
                 gamN = gb[((b + 1) & 3) * kGbFloats + 2 * kC + kC - 1];
             }
+            mbar_wait(&bars.ds_done, par, &dead, a.status);
+            tc_fence_after_sync();
+            if (last) {
+                if (a.S_T && !dead) {
 #pragma unroll 1
-            for (int q = 0; q < 4; ++q) {
-                uint32_t rr[16];
-                tmem_ld16(lane_base + kTmS + 64 * half + 16 * q, rr);
-                tmem_ld_wait();
-                if (last) {
-                    if (a.S_T) {
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t rr[16];
+                        tmem_ld16(lane_base + kTmS + 64 * half + 16 * q, rr);
+                        tmem_ld_wait();
 #pragma unroll
                         for (int c = 0; c < 16; ++c)
                             a.S_T[sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j] = __uint_as_float(rr[c]);
                     }
-                } else {
-                    float v[16];
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        v[c] = __uint_as_float(rr[c]);
-                        rr[c] = __float_as_uint(v[c] * gamN);
-                    }
-                    tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);
-                    store_row_chunks(sm + kOffSt + half * (kD * 128), j, 2 * q, v);
                 }
-            }
-            if (!last) {
+            } else {
+                uint32_t rr[4][16];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tmem_ld16(lane_base + kTmS + 64 * half + 16 * q, rr[q]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) w[e] = pack_bf16(__uint_as_float(rr[q][2 * e]), __uint_as_float(rr[q][2 * e + 1]));
+                    tmem_st8(lane_base + kTmSb + 32 * half + 8 * q, w);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) rr[q][c] = __float_as_uint(__uint_as_float(rr[q][c]) * gamN);
+                    tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr[q]);
+                }
                 tmem_st_wait();
-                fence_async_smem();
                 tc_fence_before_sync();
                 mbar_arrive(&bars.st_ready);
             }
@@ -791,24 +817,14 @@ cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s) {
     const uint64_t qk_inner = static_cast<uint64_t>(a.H_k) * kD, v_inner = static_cast<uint64_t>(a.H_v) * kD;
     if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         !make_tensor_map_2d(&mapK, a.k, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
-        (a.v && !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, kD, kC, false)) ||
+        (a.v && !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, 64, kC, true)) ||
         (a.o && !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false)))
         return cudaErrorInvalidValue;
     if (!a.v) mapV = mapK;   // never used by the kernel then
     if (!a.o) mapO = mapK;
-    // dynamic shared memory: everything the device allows beside the kernel's static part (the map needs
-    // kSmemUsed bytes from a 1024-byte aligned base; the kernel checks that it fits)
-    cudaFuncAttributes fa;
-    cudaError_t e = cudaFuncGetAttributes(&fa, gdn_scan_tensor_kernel);
+    cudaError_t e = cudaFuncSetAttribute(gdn_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    int dev = 0, optin = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
-    const int dyn = optin - static_cast<int>(fa.sharedSizeBytes);
-    if (dyn < kSmemUsed) return cudaErrorInvalidConfiguration;
-    e = cudaFuncSetAttribute(gdn_scan_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn);
-    if (e != cudaSuccess) return e;
-    gdn_scan_tensor_kernel<<<dim3(a.H_v, a.n_seq), kThreads, dyn, s>>>(a, mapQ, mapK, mapV, mapO);
+    gdn_scan_tensor_kernel<<<dim3(a.H_v, a.n_seq), kThreads, kSmemBytes, s>>>(a, mapQ, mapK, mapV, mapO);
     return cudaGetLastError();
 }
 
