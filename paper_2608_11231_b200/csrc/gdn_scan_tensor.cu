@@ -7,8 +7,8 @@
 // gam_t = e^{cg_t}, Gam_ti = e^{cg_t - cg_i}, w_t = e^{cg_C - cg_t} and S the incoming state:
 //   (1) G    = [Q;K] K^T             rows 0..63: q_t.k_i, rows 64..127: k_t.k_i           tcgen05
 //       Ps_ti = scale Gam_ti q_t.k_i (i <= t),  A_ti = beta_t Gam_ti k_t.k_i (i < t)      mask warps
-//       M    = (I + A)^{-1}          (UT transform: 16x16 diagonal blocks by substitution in fp32,
-//                                     off-diagonal blocks by tf32 block products)         prep warps
+//       M    = (I + A)^{-1}          (UT transform, by doubling: 8x8 blocks by substitution and 8 -> 16 in
+//                                     fp32, 16 -> 32 -> 64 by fp16 block products)         prep warps
 //       X_mi = M_mi beta_i           bf16 operand of the block's triangular solve          prep warps
 //  (3a) U^T  = V^T X^T               the part of the solve that does not depend on S       tcgen05
 //  (2K) KS   = S^T K^T               (S^T k_t)_j                                          tcgen05 (A = bf16 S^T in TMEM)
@@ -24,9 +24,8 @@
 // mask epilogue, the inverse, (3a), the Q scaling) runs up to two blocks ahead of the chain; (2Q) and
 // (7) hang off it.  A padded token (beyond the sequence end) has g = 0 and beta = 0: the identity step.
 //
-// Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows; they also turn the
-// finished O^T of the previous block into the output tile while (3b) runs), 8-11 mask epilogue of (1) and Q
-// scaling, 12-15 prep (the inverse), 16 TMA loads of V and the store of the output tile, 17 MMA issue of
+// Warps 0-7 chain (lane = state column, warpgroup = half of the tokens / state rows), 8-11 mask epilogue of (1)
+// and the output tile of the block the chain has finished, 12-15 prep (the inverse, Q scaling), 16 TMA loads of V and the store of the output tile, 17 MMA issue of
 // the chain, 18 TMA loads of Q and K and MMA issue of (1), 19 per-block scalars.  All waits on mbarriers
 // are bounded.
 //
@@ -34,6 +33,8 @@
 // inlined): the twenty warps run seven different programs at once, and with the first, fully unrolled
 // version of this kernel the SMs fetched a third of their instructions from the cache they share with
 // their neighbours, which then ran at 80 % of its request rate and set the pace of the whole kernel.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -71,96 +72,137 @@ constexpr uint32_t kTmS = 0;      // 128: S^T fp32
 constexpr uint32_t kTmSb = 128;   // 64: S^T as bf16 pairs (A operand of (2K), (2Q))
 constexpr uint32_t kTmKS = 192;   // 64: KS fp32; Rk as bf16 pairs in place (tokens 0..31 in columns 0..15, 32..63 in 32..47)
 constexpr uint32_t kTmU = 256;    // 64: U fp32; in place Uw as bf16 pairs (columns 0..15 and 32..47) and u (16..31 and 48..63)
-constexpr uint32_t kTmO = 320;    // 64: O^T
-constexpr uint32_t kTmG = 384;    // 2 x 64: G of the even / odd blocks
+constexpr uint32_t kTmO = 320;    // 2 x 64: O^T of the even / odd blocks
+constexpr uint32_t kTmG = 448;    // 64
 constexpr uint32_t kTmemCols = 512;
 
 struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
-    uint64_t full_qk[3], tiles_free_qk[3], full_v[2], g_done[2], ks_done, u_done, ds_done, o_mma_done, p_free[3], x_free[2];
+    uint64_t full_qk[3], tiles_free_qk[3], full_v[2], g_done[2], ks_done, u_done, ds_done, o_mma_done[4], p_free[3], x_free[2];
     // 128-thread barriers (prep or mask warpgroup)
-    uint64_t m_ready[2], qs_ready[3];
+    uint64_t m_ready[2], qs_ready[3], o_done[4], o_staged[2];
     // 64-thread barriers (the two halves of the mask warpgroup)
     uint64_t a_ready[2], p_ready[3];
     // 32-thread barriers (the scalar warp)
     uint64_t gb_ready[4];
     // 256-thread barriers (both chain warpgroups)
-    uint64_t rk_ready, uw_ready, st_ready, chain_done[4], o_done[4], o_staged[2];
+    uint64_t rk_ready, uw_ready, st_ready, chain_done[4];
 };
-constexpr int kBars1 = 19, kBars128 = 5, kBars64 = 5, kBars32 = 4, kBars256 = 13;
+constexpr int kBars1 = 22, kBars128 = 11, kBars64 = 5, kBars32 = 4, kBars256 = 7;
 static_assert(sizeof(Bars) == 8 * (kBars1 + kBars128 + kBars64 + kBars32 + kBars256), "barrier table");
 
-__device__ __forceinline__ uint32_t to_tf32(float v) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(v));
-    return r;
-}
-// acc[16 x 8] += A[16 x 8] B[8 x 8] on the warp-level MMA; fragments as the PTX ISA lays them out
-// (row = lane / 4 (+8), column = lane % 4 (+4) for A; k = lane % 4 (+4), n = lane / 4 for B; row = lane / 4 (+8),
-// columns 2 (lane % 4), +1 for the accumulator).
-__device__ __forceinline__ void mma_tf32_16x8x8(float (&acc)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+// Warp-level tensor-core MMA on fp16 operands (11-bit significands like tf32, but 16 k-elements per
+// instruction): acc[16 x 8] += A[16 x 16] B[16 x 8], fp32 accumulation.  Fragments as the PTX ISA lays them out.
+// Every operand here is an entry of A or of an inverse of I + A: of order one or smaller, far inside the fp16 range.
+__device__ __forceinline__ void mma_f16_16x8x16(float (&acc)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
         : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+// A operand: the 16 x 16 tile at p of a row-major fp32 matrix (row stride kLd); gid = lane / 4, tig = lane % 4
+__device__ __forceinline__ void frag_a(uint32_t (&a)[4], const float *p, int gid, int tig) {
+    const float2 v0 = *reinterpret_cast<const float2 *>(p + gid * kLd + 2 * tig);
+    const float2 v1 = *reinterpret_cast<const float2 *>(p + (gid + 8) * kLd + 2 * tig);
+    const float2 v2 = *reinterpret_cast<const float2 *>(p + gid * kLd + 2 * tig + 8);
+    const float2 v3 = *reinterpret_cast<const float2 *>(p + (gid + 8) * kLd + 2 * tig + 8);
+    a[0] = pack_f16(v0.x, v0.y); a[1] = pack_f16(v1.x, v1.y); a[2] = pack_f16(v2.x, v2.y); a[3] = pack_f16(v3.x, v3.y);
+}
+// B operand: the 16 (k) x 8 (n) tile at p of a row-major fp32 matrix B[k][n]
+__device__ __forceinline__ void frag_b(uint32_t &b0, uint32_t &b1, const float *p, int gid, int tig) {
+    b0 = pack_f16(p[(2 * tig) * kLd + gid], p[(2 * tig + 1) * kLd + gid]);
+    b1 = pack_f16(p[(2 * tig + 8) * kLd + gid], p[(2 * tig + 9) * kLd + gid]);
+}
+// accumulator tile [16 x 8] -> p (row-major fp32), times sgn
+__device__ __forceinline__ void store_acc(float *p, const float (&acc)[4], float sgn, int gid, int tig) {
+    *reinterpret_cast<float2 *>(p + gid * kLd + 2 * tig) = make_float2(sgn * acc[0], sgn * acc[1]);
+    *reinterpret_cast<float2 *>(p + (gid + 8) * kLd + 2 * tig) = make_float2(sgn * acc[2], sgn * acc[3]);
 }
 
-// One off-diagonal block (r = c + D, c) of M = (I + A)^{-1}, or NH = 1 half of it (8 columns from 8 nh0):
-// X = sum_{m=c}^{r-1} A_rm M_mc, M_rc = -D_r X with D_r the inverted diagonal block.  tf32 operands rounded to
-// nearest, fp32 accumulation.  Every MMA of a stage has its own accumulator, so they are all in flight together
-// (the warp-level MMA has a long latency here); X passes through the unused block (c, r) above the diagonal to
-// change from accumulator to operand layout.  A, M: fp32 [64][ld].
-template <int NH, int D>
-__device__ __forceinline__ void inv_offdiag(const float *Af, float *Mf, int c, int nh0, int gid, int tig) {
-    constexpr int ld = kLd;
-    const int r = c + D;
-    float part[D][2][NH][4];
+// The inverse M = (I + A)^{-1} of the unit lower triangular 64x64 matrix of a block is built by doubling:
+// 8x8 diagonal blocks by forward substitution, then three merges
+//     inv [[L1, 0], [A21, L2]] = [[inv L1, 0], [-inv(L2) A21 inv(L1), inv L2]]
+// from 8 to 16 (fp32 FMAs), 16 to 32 and 32 to 64 (warp-level tensor-core MMA, fp16 operands rounded to nearest,
+// fp32 accumulation): four rounds of dependent MMAs per block, eight MMAs per warp in all.
+// A, M: fp32 [64][kLd]; the part of M above the block diagonal serves as scratch.
+//
+// 16 -> 32: half (8 columns from 8 nh) of the 16x16 block (c + 1, c): X = A_rc M_cc, M_rc = -M_rr X; X passes
+// through the unused block (c, r) above the diagonal to change from accumulator to operand layout.
+__device__ __forceinline__ void inv_merge32(const float *Af, float *Mf, int c, int nh, int gid, int tig) {
+    const int r = c + 1;
+    uint32_t a[4], b0, b1;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    frag_a(a, Af + (16 * r) * kLd + 16 * c, gid, tig);
+    frag_b(b0, b1, Mf + (16 * c) * kLd + 16 * c + 8 * nh, gid, tig);
+    mma_f16_16x8x16(acc, a, b0, b1);
+    float *xs = Mf + (16 * c) * kLd + 16 * r + 8 * nh;
+    store_acc(xs, acc, 1.f, gid, tig);
+    __syncwarp();
 #pragma unroll
-    for (int mm = 0; mm < D; ++mm) {
+    for (int i = 0; i < 4; ++i) acc[i] = 0.f;
+    frag_a(a, Mf + (16 * r) * kLd + 16 * r, gid, tig);
+    frag_b(b0, b1, xs, gid, tig);
+    mma_f16_16x8x16(acc, a, b0, b1);
+    store_acc(Mf + (16 * r) * kLd + 16 * c + 8 * nh, acc, -1.f, gid, tig);
+}
+// 32 -> 64, first half: T = A21 inv(L1) with A21 = A[32.., 0..31], inv(L1) = M[0..31, 0..31] (lower triangular by 16x16
+// blocks).  Warp (mt, nb) computes rows 16 mt .. +15, columns 16 nb .. +15 of T into the scratch M[0..31, 32..63].
+__device__ __forceinline__ void inv_merge64_a(const float *Af, float *Mf, int mt, int nb, int gid, int tig) {
+    float acc[2][2][4];
 #pragma unroll
-        for (int ks = 0; ks < 2; ++ks) {
-            const float *ap = Af + (16 * r + gid) * ld + 16 * (c + mm) + 8 * ks + tig;
-            const uint32_t a0 = to_tf32(ap[0]), a1 = to_tf32(ap[8 * ld]), a2 = to_tf32(ap[4]), a3 = to_tf32(ap[8 * ld + 4]);
+    for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-            for (int hh = 0; hh < NH; ++hh) {
-                const float *bp = Mf + (16 * (c + mm) + 8 * ks + tig) * ld + 16 * c + 8 * (nh0 + hh) + gid;
+        for (int e = 0; e < 2; ++e)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) part[mm][ks][hh][i] = 0.f;
-                mma_tf32_16x8x8(part[mm][ks][hh], a0, a1, a2, a3, to_tf32(bp[0]), to_tf32(bp[4 * ld]));
+            for (int i = 0; i < 4; ++i) acc[nt][e][i] = 0.f;
+#pragma unroll
+    for (int kb = 0; kb < 2; ++kb) {
+        if (kb >= nb) {   // rows of inv(L1) above its block diagonal are zero
+            uint32_t a[4], b0, b1;
+            frag_a(a, Af + (32 + 16 * mt) * kLd + 16 * kb, gid, tig);
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                frag_b(b0, b1, Mf + (16 * kb) * kLd + 16 * nb + 8 * nt, gid, tig);
+                mma_f16_16x8x16(acc[nt][kb], a, b0, b1);
             }
         }
     }
-    float *xs = Mf + (16 * c) * ld + 16 * r + 8 * nh0;
 #pragma unroll
-    for (int hh = 0; hh < NH; ++hh) {
-        float x[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-        for (int mm = 0; mm < D; ++mm)
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) x[i] += part[mm][ks][hh][i];
-        *reinterpret_cast<float2 *>(xs + 8 * hh + gid * ld + 2 * tig) = make_float2(x[0], x[1]);
-        *reinterpret_cast<float2 *>(xs + 8 * hh + (gid + 8) * ld + 2 * tig) = make_float2(x[2], x[3]);
+        for (int i = 0; i < 4; ++i) acc[nt][0][i] += acc[nt][1][i];
+        store_acc(Mf + (16 * mt) * kLd + 32 + 16 * nb + 8 * nt, acc[nt][0], 1.f, gid, tig);
     }
-    __syncwarp();
-    float out[2][NH][4];
+}
+// 32 -> 64, second half: M[32.., 0..31] = -inv(L2) T with inv(L2) = M[32.., 32..] (lower triangular by blocks).
+__device__ __forceinline__ void inv_merge64_b(float *Mf, int mt, int nb, int gid, int tig) {
+    float acc[2][2][4];
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks) {
-        const float *dp = Mf + (16 * r + gid) * ld + 16 * r + 8 * ks + tig;
-        const uint32_t a0 = to_tf32(dp[0]), a1 = to_tf32(dp[8 * ld]), a2 = to_tf32(dp[4]), a3 = to_tf32(dp[8 * ld + 4]);
+    for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
-        for (int hh = 0; hh < NH; ++hh) {
-            const float *xp = xs + 8 * hh + (8 * ks + tig) * ld + gid;
+        for (int e = 0; e < 2; ++e)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) out[ks][hh][i] = 0.f;
-            mma_tf32_16x8x8(out[ks][hh], a0, a1, a2, a3, to_tf32(xp[0]), to_tf32(xp[4 * ld]));
+            for (int i = 0; i < 4; ++i) acc[nt][e][i] = 0.f;
+#pragma unroll
+    for (int kb = 0; kb < 2; ++kb) {
+        if (kb <= mt) {   // columns of inv(L2) right of its block diagonal are zero
+            uint32_t a[4], b0, b1;
+            frag_a(a, Mf + (32 + 16 * mt) * kLd + 32 + 16 * kb, gid, tig);
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                frag_b(b0, b1, Mf + (16 * kb) * kLd + 32 + 16 * nb + 8 * nt, gid, tig);
+                mma_f16_16x8x16(acc[nt][kb], a, b0, b1);
+            }
         }
     }
 #pragma unroll
-    for (int hh = 0; hh < NH; ++hh) {
-        float *mp = Mf + (16 * r + gid) * ld + 16 * c + 8 * (nh0 + hh) + 2 * tig;
-        *reinterpret_cast<float2 *>(mp) = make_float2(-(out[0][hh][0] + out[1][hh][0]), -(out[0][hh][1] + out[1][hh][1]));
-        *reinterpret_cast<float2 *>(mp + 8 * ld) = make_float2(-(out[0][hh][2] + out[1][hh][2]), -(out[0][hh][3] + out[1][hh][3]));
+    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nt][0][i] += acc[nt][1][i];
+        store_acc(Mf + (32 + 16 * mt) * kLd + 16 * nb + 8 * nt, acc[nt][0], -1.f, gid, tig);
     }
 }
 __device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
@@ -363,10 +405,10 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     tma_load_2d(base + kb * 2 * kC * 128, &mapQ, hk * kD + kb * 64, row, &bars.full_qk[s3]);
                     tma_load_2d(base + kb * 2 * kC * 128 + kC * 128, &mapK, hk * kD + kb * 64, row, &bars.full_qk[s3]);
                 }
-                // (1) of block b: the mask epilogue of block b-2 has drained these G columns
-                if (b >= 2) {
-                    mbar_wait(&bars.a_ready[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-                    mbar_wait(&bars.p_ready[(b - 2) % 3], ((b - 2) / 3) & 1, &dead, a.status);
+                // (1) of block b: the mask epilogue of block b-1 has drained the G columns
+                if (b >= 1) {
+                    mbar_wait(&bars.a_ready[(b - 1) & 1], ((b - 1) >> 1) & 1, &dead, a.status);
+                    mbar_wait(&bars.p_ready[(b - 1) % 3], ((b - 1) / 3) & 1, &dead, a.status);
                 }
                 mbar_wait(&bars.full_qk[s3], (b / kQKStages) & 1, &dead, a.status);
                 tc_fence_after_sync();
@@ -374,7 +416,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll 1
                 for (int k = 0; k < 8; ++k) {
                     const uint64_t off = ((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4;
-                    umma_bf16(tm + kTmG + 64 * (b & 1), dQK + off, dQK + off + ((kC * 128) >> 4), idG, k > 0);
+                    umma_bf16(tm + kTmG, dQK + off, dQK + off + ((kC * 128) >> 4), idG, k > 0);
                 }
                 umma_commit(&bars.g_done[b & 1]);
             }
@@ -399,6 +441,16 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int k = 0; k < 8; ++k)
                     umma_bf16_ts(tm + kTmKS, tm + kTmSb + 8 * k, dK + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
                 umma_commit(&bars.ks_done);
+                // (2Q) O = S^T Qs^T right behind (2K), off the chain: it reads the same bf16 state; the O columns of this
+                // parity were drained with the outputs of block b-2
+                if (has_o) {
+                    if (b >= 2) mbar_wait(&bars.o_done[(b - 2) & 3], ((b - 2) >> 2) & 1, &dead, a.status);
+                    mbar_wait(&bars.qs_ready[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16_ts(tm + kTmO + 64 * par, tm + kTmSb + 8 * k, dQ + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
+                }
                 // (3a) U = V^T X^T: needs the inverse of the block and the V tile (the U columns were read by (5) and (7)
                 // of the previous block, issued before)
                 mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
@@ -417,16 +469,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     umma_bf16_ts(tm + kTmU, tm + kTmKS + 32 * (k >> 1) + 8 * (k & 1), dX + 2 * k, idN64, has_v || k > 0);
                 umma_commit(&bars.u_done);
                 umma_commit(&bars.x_free[b & 1]);
-                // (2Q) O = S^T Qs^T behind (3b): the chain warps drain the O columns of the previous block while (3b)
-                // runs, before they turn to U, so this wait never outlasts the next one
-                if (has_o) {
-                    if (b > 0) mbar_wait(&bars.o_done[(b - 1) & 3], ((b - 1) >> 2) & 1, &dead, a.status);
-                    mbar_wait(&bars.qs_ready[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        umma_bf16_ts(tm + kTmO, tm + kTmSb + 8 * k, dQ + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
-                }
                 // (5) accumulates onto the pre-scaled state; B = K tile read MN-major (rows = tokens)
                 mbar_wait(&bars.uw_ready, par, &dead, a.status);
                 tc_fence_after_sync();
@@ -443,10 +485,10 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     const uint64_t dP = umma_desc(smem_u32(sm + kOffP + (b % 3) * (kC * 128)), 0, 1024);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        umma_bf16_ts(tm + kTmO, tm + kTmU + 32 * (k >> 1) + 16 + 8 * (k & 1), dP + 2 * k, idN64, true);
+                        umma_bf16_ts(tm + kTmO + 64 * par, tm + kTmU + 32 * (k >> 1) + 16 + 8 * (k & 1), dP + 2 * k, idN64, true);
                     umma_commit(&bars.p_free[b % 3]);
                 }
-                umma_commit(&bars.o_mma_done);
+                umma_commit(&bars.o_mma_done[b & 3]);
             }
         }
     } else if (warp >= 12) {
@@ -460,17 +502,17 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.a_ready[b & 1], (b >> 1) & 1, &dead, a.status);
             named_bar_sync(1, 128);   // every thread is done with the fp32 M of the previous block
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
-            // ---- M = (I + A)^{-1}.  Diagonal 16x16 blocks: thread (k, c) solves column c of block k by forward
-            // substitution; each row of the block is fetched with four 16-byte loads ahead of its use.
+            // ---- M = (I + A)^{-1} by doubling.  8x8 diagonal blocks: thread (k, c) solves column c of block k by forward
+            // substitution (fp32).
             if (x < kC) {
-                const int k = x >> 4, c = x & 15;
-                const float *Ab = Af + (16 * k) * kLd + 16 * k;
-                float xv[16];
+                const int k = x >> 3, c = x & 7;
+                const float *Ab = Af + (8 * k) * kLd + 8 * k;
+                float xv[8];
 #pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    float row[16];
+                for (int t = 0; t < 8; ++t) {
+                    float row[8];
 #pragma unroll
-                    for (int i4 = 0; i4 < 16; i4 += 4) {
+                    for (int i4 = 0; i4 < 8; i4 += 4) {
                         if (i4 < t) {
                             const float4 v = *reinterpret_cast<const float4 *>(Ab + t * kLd + i4);
                             row[i4] = v.x; row[i4 + 1] = v.y; row[i4 + 2] = v.z; row[i4 + 3] = v.w;
@@ -485,18 +527,47 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     xv[t] = (t >= c) ? acc0 + acc1 : 0.f;
                 }
 #pragma unroll
-                for (int t = 0; t < 16; ++t) Mf[(16 * k + t) * kLd + 16 * k + c] = xv[t];
+                for (int t = 0; t < 8; ++t) Mf[(8 * k + t) * kLd + 8 * k + c] = xv[t];
             }
             named_bar_sync(1, 128);
-            // Off-diagonal blocks by distance d from the diagonal, M_rc = -D_r sum_{m=c}^{r-1} A_rm M_mc, on the
-            // warp-level tensor-core MMA; one warp per block (d = 1) or half block (d = 2, 3).
+            // 8 -> 16 in fp32: thread = (16-block k, row i, column pair) of the 8x8 block below the diagonal;
+            // T = A21 inv(L1) passes through the scratch M[0..31, 32..39]
+            {
+                const int k = x >> 5, i = (x >> 2) & 7, j0 = 2 * (x & 3);
+                const float *a21 = Af + (16 * k + 8 + i) * kLd + 16 * k;
+                const float *d1 = Mf + (16 * k) * kLd + 16 * k;
+                float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    const float av = a21[m];
+                    t0 = fmaf(av, d1[m * kLd + j0], t0);        // zero where m < j: inv(L1) is lower triangular
+                    t1 = fmaf(av, d1[m * kLd + j0 + 1], t1);
+                }
+                float *ts = Mf + (8 * k) * kLd + 32;
+                *reinterpret_cast<float2 *>(ts + i * kLd + j0) = make_float2(t0, t1);
+                named_bar_sync(1, 128);
+                const float *d2 = Mf + (16 * k + 8 + i) * kLd + 16 * k + 8;
+                float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    const float dv = d2[m];                       // zero where m > i
+                    m0 = fmaf(dv, ts[m * kLd + j0], m0);
+                    m1 = fmaf(dv, ts[m * kLd + j0 + 1], m1);
+                }
+                *reinterpret_cast<float2 *>(Mf + (16 * k + 8 + i) * kLd + 16 * k + j0) = make_float2(-m0, -m1);
+                // the 8x8 block above the diagonal of the 16x16 block reads as part of the operands later: zero
+                *reinterpret_cast<float2 *>(Mf + (16 * k + i) * kLd + 16 * k + 8 + j0) = make_float2(0.f, 0.f);
+            }
+            named_bar_sync(1, 128);
             {
                 const int wq = warp & 3, gid = lane >> 2, tig = lane & 3;
-                if (wq < 3) inv_offdiag<2, 1>(Af, Mf, wq, 0, gid, tig);
+                // 16 -> 32: blocks (1, 0) and (3, 2), one half block per warp
+                inv_merge32(Af, Mf, 2 * (wq >> 1), wq & 1, gid, tig);
                 named_bar_sync(1, 128);
-                inv_offdiag<1, 2>(Af, Mf, wq >> 1, wq & 1, gid, tig);
+                // 32 -> 64: one 16x16 block of the 32x32 result per warp
+                inv_merge64_a(Af, Mf, wq >> 1, wq & 1, gid, tig);
                 named_bar_sync(1, 128);
-                if (wq < 2) inv_offdiag<1, 3>(Af, Mf, 0, wq, gid, tig);
+                inv_merge64_b(Mf, wq >> 1, wq & 1, gid, tig);
                 named_bar_sync(1, 128);
             }
             // ---- X = M diag(beta) as bf16 operand (zeros above the block diagonal); the buffer of this parity was
@@ -522,6 +593,24 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             }
             fence_async_smem();
             mbar_arrive(&bars.m_ready[b & 1]);
+            // ---- Q tile of block b scaled in place by scale gam_t ((1) has read it: its result was masked before the
+            // inverse began): thread = (token, 64-column half)
+            if (has_o) {
+                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);   // this thread reads what the TMA wrote
+                unsigned char *qt = sm + (b % kQKStages) * kQKStage + (x >> 6) * (2 * kC * 128) + (x & 63) * 128;
+                const __nv_bfloat162 f2 = __float2bfloat162_rn(a.scale * sc[2 * kC + (x & 63)]);
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    uint4 *p = reinterpret_cast<uint4 *>(qt + ((c ^ (x & 7)) << 4));
+                    uint4 v = *p;
+                    __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) e[i] = __hmul2(e[i], f2);
+                    *p = v;
+                }
+                fence_async_smem();
+                mbar_arrive(&bars.qs_ready[b % kQKStages]);
+            }
         }
     } else if (warp >= 8) {
         // ======================================================= mask warpgroup: epilogue of (1) and Q scaling, as far ahead of the
@@ -548,8 +637,42 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
             }
         }
+        // outputs of block b: O^T (complete once (7) has run) -> bf16 tile [token][j], lane = j
+        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
+        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
+        auto o_epilogue = [&](int b) {
+            mbar_wait(&bars.o_mma_done[b & 3], (b >> 2) & 1, &dead, a.status);
+            tc_fence_after_sync();
+            const int t0 = t_begin + b * kC;
+            const int n = min(kC, t_end - t0);
+            if (has_o && (n == kC || !dead)) {
+                // whole block: stage the tile in the V stage of this block, which (3a) has finished reading; the
+                // store warp writes it out with TMA
+                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffV + (b & 1) * kVStage) + x;
 #pragma unroll 1
-        for (int b = 0; b < nblk; ++b) {
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t taddr = lane_base + kTmO + 64 * (b & 1) + 16 * q;
+                    if (n != kC) {
+                        store_o_partial(taddr, o + (static_cast<size_t>(t0 + 16 * q) * a.H_v + h) * kD + x, tstride, n - 16 * q);
+                        continue;
+                    }
+                    uint32_t pu[16];
+                    tmem_ld16(taddr, pu);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) os[(16 * q + c) * kD] = __float2bfloat16_rn(__uint_as_float(pu[c]));
+                }
+                fence_async_smem();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bars.o_done[b & 3]);
+            mbar_arrive(&bars.o_staged[b & 1]);
+        };
+#pragma unroll 1
+        for (int b = 0; b < nblk + 3; ++b) {
+            // the outputs lag the masks by three blocks: by then the chain has normally produced them
+            if (b >= 3) o_epilogue(b - 3);
+            if (b >= nblk) continue;
             const float *sc = gb + (b & 3) * kGbFloats;
             mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
             float *Af = reinterpret_cast<float *>(sm + kOffA) + (b & 1) * (kC * kLd);
@@ -570,7 +693,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 const float coef = (x < kC) ? a.scale : sc[kC + t];     // rows of Ps: the output scale, rows of A: beta_t
                 const int lim = (x < kC) ? t : t - 1;                   // P keeps the diagonal, A is strictly lower
                 const bool fast = sc[5 * kC] + sc[5 * kC + 1] == 0.f;
-                const uint32_t tmg = lane_base + kTmG + 64 * (b & 1);
+                const uint32_t tmg = lane_base + kTmG;
                 // column groups above the diagonal for every row of this warp are never touched
 #pragma unroll 1
                 for (int q = 0; 16 * q <= row_hi; ++q) {
@@ -586,13 +709,25 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     float aa;
                     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(aa) : "f"(fminf(cgt - sc[i0], 0.f)));
                     aa *= coef;
+                    if (i0 + 15 <= row_hi - 32) {
+                        // below the diagonal for every row of this warp: no masking
 #pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                        v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
-                        v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
-                        v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
-                        v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                        for (int c = 0; c < 16; c += 4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                            v[c] = __uint_as_float(rr[c]) * aa * f.x;
+                            v[c + 1] = __uint_as_float(rr[c + 1]) * aa * f.y;
+                            v[c + 2] = __uint_as_float(rr[c + 2]) * aa * f.z;
+                            v[c + 3] = __uint_as_float(rr[c + 3]) * aa * f.w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 16; c += 4) {
+                            const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
+                            v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
+                            v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
+                            v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
+                            v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                        }
                     }
                     if (x < kC) {
                         store_row_chunks(ps, t, 2 * q, v);
@@ -610,30 +745,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             } else {
                 mbar_arrive(&bars.a_ready[b & 1]);
             }
-            // Q tile of block b scaled in place by scale gam_t now that (1) has read it: thread = (token, 64-column half)
-            if (has_o) {
-                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);   // this thread reads what the TMA wrote
-                unsigned char *qt = sm + (b % kQKStages) * kQKStage + (x >> 6) * (2 * kC * 128) + t * 128;
-                const __nv_bfloat162 f2 = __float2bfloat162_rn(a.scale * sc[2 * kC + t]);
-#pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
-                    uint4 *p = reinterpret_cast<uint4 *>(qt + ((c ^ (t & 7)) << 4));
-                    uint4 v = *p;
-                    __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) e[i] = __hmul2(e[i], f2);
-                    *p = v;
-                }
-                fence_async_smem();
-                mbar_arrive(&bars.qs_ready[b % kQKStages]);
-            }
         }
     } else {
         // ======================================================= chain warpgroups: lane = state column j, `half` = token / row half
         const int j = tid & 127, half = warp >> 2;
         const uint32_t lane_base = tm + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(a.o);
-        const size_t tstride = static_cast<size_t>(a.H_v) * kD;
         // initial state: S0[m][j], m = 64*half..+63 -> TMEM (fp32, pre-scaled by gam_C of block 0) and bf16 pairs
         mbar_wait(&bars.gb_ready[0], 0, &dead, a.status);
         {
@@ -656,41 +772,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tc_fence_before_sync();
             mbar_arrive(&bars.st_ready);
         }
-        // outputs of block b: O^T (complete once (7) has run) -> bf16 tile, tokens 32*half..+31
-        auto o_epilogue = [&](int b) {
-            mbar_wait(&bars.o_mma_done, b & 1, &dead, a.status);
-            tc_fence_after_sync();
-            const int t0 = t_begin + b * kC;
-            const int n = min(kC, t_end - t0);
-            if (has_o && (n == kC || !dead)) {
-                // whole block: stage the tile [token][j] in the V stage of this block, which (3a) has finished
-                // reading; the store warp writes it out with TMA
-                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffV + (b & 1) * kVStage) + (32 * half) * kD + j;
 #pragma unroll 1
-                for (int q = 0; q < 2; ++q) {
-                    const uint32_t taddr = lane_base + kTmO + 32 * half + 16 * q;
-                    if (n != kC) {
-                        store_o_partial(taddr, o + (static_cast<size_t>(t0 + 32 * half + 16 * q) * a.H_v + h) * kD + j, tstride, n - 32 * half - 16 * q);
-                        continue;
-                    }
-                    uint32_t pu[16];
-                    tmem_ld16(taddr, pu);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int c = 0; c < 16; ++c) os[(16 * q + c) * kD] = __float2bfloat16_rn(__uint_as_float(pu[c]));
-                }
-                fence_async_smem();
-            }
-            tc_fence_before_sync();
-            mbar_arrive(&bars.o_done[b & 3]);
-            mbar_arrive(&bars.o_staged[b & 1]);
-        };
-#pragma unroll 1
-        for (int b = 0; b <= nblk; ++b) {
-            if (b == nblk) {   // the outputs of the last block
-                o_epilogue(b - 1);
-                break;
-            }
+        for (int b = 0; b < nblk; ++b) {
             const uint32_t par = b & 1;
             const float *sc = gb + (b & 3) * kGbFloats;
             if (b > 0) mbar_wait(&bars.gb_ready[b & 3], (b >> 2) & 1, &dead, a.status);
@@ -721,8 +804,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(&bars.rk_ready);
-            // while (3b) runs: the outputs of the previous block
-            if (b > 0) o_epilogue(b - 1);
             // u_t[j], tokens 32*half..+31 -> Uw = w o u as bf16 pairs over the first 16 of this thread's own 32 columns, u over the rest
             mbar_wait(&bars.u_done, par, &dead, a.status);
             tc_fence_after_sync();
