@@ -24,6 +24,12 @@
  *     int32 arrays: they are range-checked on the host before anything is
  *     launched and copied to the device by the call itself (into the
  *     caller's workspace).  They may be reused as soon as the call returns.
+ *     A list that fits the kernel parameters (n_req + 1 + selection indices +
+ *     chunk ids <= 4000 ints for the initialisers, n_seq + 1 <= 1000 for the
+ *     scans) travels inside the launch and the call may be captured into a
+ *     CUDA graph; a longer list needs a host-to-device copy of an array that
+ *     dies with the call, so such a call returns LKV_ERR_UNSUPPORTED while
+ *     `stream` is capturing.
  *   - The caller owns every buffer.  The library allocates nothing, frees
  *     nothing and keeps no pointer after a call returns; scratch lives in a
  *     caller-provided workspace whose size lkv_workspace_bytes() reports.
@@ -35,11 +41,17 @@
  *     that case.  There is no CPU fallback: an unsupported shape returns
  *     LKV_ERR_UNSUPPORTED.
  *   - Device-side waits (TMA / tensor-core completion barriers) are bounded.
- *     A kernel that gives up sets the status word at the start of the
- *     workspace and returns; lkv_device_status() reads it.
+ *     A kernel whose wait runs out sets the status word (the first 4 bytes of
+ *     the workspace), drains without writing any further result, and returns;
+ *     lkv_device_status() reads the word.  The word is sticky: the library
+ *     only ever sets it.  The caller zeroes the first 256 bytes of a
+ *     workspace once before its first use, and again after a reported
+ *     time-out; results of a call whose workspace reports a time-out are
+ *     undefined (partly written).
  *   - Data pointers must be 16-byte aligned (LKV_ERR_ALIGN otherwise).
- *   - Outputs must not overlap inputs, except that S_T may be the same buffer
- *     as S0 in the scan calls.
+ *   - Outputs must not overlap inputs or each other (LKV_ERR_OVERLAP, checked
+ *     on the host from the sizes the descriptor implies), except that S_T
+ *     may be exactly S0 in the scan calls.
  *   - States are row-major [.., d_k, d_v] with d_v contiguous, always fp32 on
  *     output.  All results are deterministic: the same inputs give the same
  *     bits on every run.
@@ -67,6 +79,7 @@ extern "C" {
 #define LKV_ERR_WORKSPACE (-7)      /* workspace missing or too small */
 #define LKV_ERR_CUDA (-8)           /* a CUDA runtime call failed (launch, copy, attribute) */
 #define LKV_ERR_DEVICE_TIMEOUT (-9) /* a bounded device-side wait ran out (reported by lkv_device_status) */
+#define LKV_ERR_OVERLAP (-10)       /* an output buffer overlaps an input buffer or another output */
 
 /* recurrence family (Eq. 2 vs Eq. 3) */
 #define LKV_FAMILY_MAMBA2 0
@@ -225,6 +238,10 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
  *     runs.  Two calls that can overlap on the GPU (different streams, no ordering
  *     between them) race on it: order them, or use lkv_init_state_batched with
  *     separate workspaces.
+ *   - The status word of a bounded device-side wait lives in the same array (it
+ *     starts at zero when the library is loaded).  The caller has no pointer to it:
+ *     lkv_device_status_static() reads it, and clears it when it was set.
+ *   - An argument error is found before anything is put on the stream.
  *   - Everything else (arguments, modes, errors, results) is as for
  *     lkv_init_state_batched; results are identical bit for bit.
  */
@@ -233,6 +250,12 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
 int lkv_init_state_batched_static(const void *states, const void *transitions, const int32_t *chunk_ids,
                                   const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index,
                                   void *S0, const lkv_init_desc *d, void *stream);
+/*
+ * Status word of the scratch of lkv_init_state_batched_static on the current device: synchronises
+ * `stream`, returns LKV_OK or LKV_ERR_DEVICE_TIMEOUT, and resets the word after reporting a time-out
+ * (LKV_ERR_CUDA if a runtime call fails).  Allocates nothing.  (No counterpart in the paper.)
+ */
+int lkv_device_status_static(void *stream);
 
 /*
  * Gated DeltaNet scan from an initial state (Eq. 1 with Eq. 3; Algorithm 1, line 3).
@@ -309,6 +332,16 @@ size_t lkv_workspace_bytes(int which, const void *desc, int n_units, int n_index
  * The only call here that blocks the host.
  */
 int lkv_device_status(const void *workspace, void *stream);
+
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper): launches one small kernel that
+ * waits, with the wait every tensor-core kernel of the library uses, on a barrier nobody will ever arrive on,
+ * giving up after `poll_limit` polls (1 .. 2^20).  The kernel then sets the status word of `workspace`
+ * (device, 16-byte aligned, at least 256 bytes, zeroed by the caller) and ends; it neither traps nor spins on.
+ * Afterwards lkv_device_status(workspace) must report LKV_ERR_DEVICE_TIMEOUT, and word 1 of the workspace
+ * must still be zero (it is set if a wait claimed to have succeeded).
+ */
+int lkv_selftest_bounded_wait(int poll_limit, void *workspace, void *stream);
 
 /* Human-readable name of a status code (static storage, never NULL). */
 const char *lkv_status_string(int status);

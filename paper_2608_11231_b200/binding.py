@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "liblkv.so")
 # constants of include/lkv.h
 LKV_OK = 0
 LKV_ERR_NULL, LKV_ERR_DIM, LKV_ERR_MODE, LKV_ERR_INDEX, LKV_ERR_ALIGN = -1, -2, -3, -4, -5
-LKV_ERR_UNSUPPORTED, LKV_ERR_WORKSPACE, LKV_ERR_CUDA, LKV_ERR_DEVICE_TIMEOUT = -6, -7, -8, -9
+LKV_ERR_UNSUPPORTED, LKV_ERR_WORKSPACE, LKV_ERR_CUDA, LKV_ERR_DEVICE_TIMEOUT, LKV_ERR_OVERLAP = -6, -7, -8, -9, -10
 LKV_FAMILY_MAMBA2, LKV_FAMILY_GDN = 0, 1
 LKV_DTYPE_F32, LKV_DTYPE_BF16 = 0, 1
 LKV_INIT_LAST, LKV_INIT_INDEX, LKV_INIT_EXACT = 0, 1, 2
@@ -29,7 +29,8 @@ LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
            "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_state_rel_error",
-           "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_status_string", "lkv_version")
+           "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_device_status_static",
+           "lkv_selftest_bounded_wait", "lkv_status_string", "lkv_version")
 
 
 class lkv_init_desc(ctypes.Structure):
@@ -85,10 +86,12 @@ def load() -> ctypes.CDLL:
         lib.lkv_workspace_bytes.argtypes = [ci, vp, ci, ci]
         lib.lkv_workspace_bytes.restype = ctypes.c_size_t
         lib.lkv_device_status.argtypes = [vp, vp]
+        lib.lkv_device_status_static.argtypes = [vp]
+        lib.lkv_selftest_bounded_wait.argtypes = [ci, vp, vp]
         lib.lkv_status_string.argtypes = [ci]
         lib.lkv_status_string.restype = ctypes.c_char_p
         for name in ("lkv_init_state", "lkv_init_state_batched", "lkv_gdn_fwd", "lkv_ssd_fwd",
-                     "lkv_device_status", "lkv_version"):
+                     "lkv_device_status", "lkv_device_status_static", "lkv_selftest_bounded_wait", "lkv_version"):
             getattr(lib, name).restype = ci
         _lib = lib
     return _lib
@@ -154,6 +157,16 @@ def lkv_workspace_bytes(which: int, desc, n_units: int, n_index: int = 0) -> int
 
 def lkv_device_status(ws: torch.Tensor, stream=None) -> int:
     return int(load().lkv_device_status(_ptr(ws), _stream(stream)))
+
+
+def lkv_device_status_static(stream=None) -> int:
+    """Status of the scratch of lkv_init_state_batched_static on the current device (cleared after a time-out)."""
+    return int(load().lkv_device_status_static(_stream(stream)))
+
+
+def lkv_selftest_bounded_wait(poll_limit: int, ws: torch.Tensor, stream=None) -> int:
+    """Launches the kernel whose only job is to let a bounded wait run out; the status word of ws is set."""
+    return int(load().lkv_selftest_bounded_wait(int(poll_limit), _ptr(ws), _stream(stream)))
 
 
 def _init_desc(states, family, compute, ws_t, n_units, n_index, chunk_ids_np=None, sel_index=0):

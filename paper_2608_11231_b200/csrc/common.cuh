@@ -108,4 +108,7 @@ int state_err_parts(size_t elems);
 cudaError_t launch_state_rel_error(const float *x, const float *r, float *rel_err, int n_states, size_t elems,
                                    float *partials, cudaStream_t s);
 
+// one CTA waits on an mbarrier nobody arrives on, with the kernels' own bounded wait and a small poll limit
+cudaError_t launch_selftest_bounded_wait(uint32_t poll_limit, int32_t *status, cudaStream_t s);
+
 }  // namespace lkv

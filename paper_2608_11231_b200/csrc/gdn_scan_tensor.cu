@@ -34,6 +34,7 @@
 // version of this kernel the SMs fetched a third of their instructions from the cache they share with
 // their neighbours, which then ran at 80 % of its request rate and set the pace of the whole kernel.
 #include <cuda_fp16.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "tc_common.cuh"
@@ -267,7 +268,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ Bars bars;
     __shared__ uint32_t tmem_base;
-    __shared__ int dead;
+    __shared__ volatile int dead;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, seq = blockIdx.y;
@@ -896,7 +897,12 @@ cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s) {
     CUtensorMap mapQ, mapK, mapV, mapO;
     const uint64_t rows = static_cast<uint64_t>(a.T_total);
     const uint64_t qk_inner = static_cast<uint64_t>(a.H_k) * kD, v_inner = static_cast<uint64_t>(a.H_v) * kD;
-    if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
+    if (rows == 0) {
+        // no token anywhere: every CTA hands its state through and never touches a tile (and a map of zero rows
+        // cannot be encoded)
+        memset(&mapQ, 0, sizeof(mapQ));
+        mapK = mapV = mapO = mapQ;
+    } else if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         !make_tensor_map_2d(&mapK, a.k, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         (a.v && !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, 64, kC, true)) ||
         (a.o && !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false)))

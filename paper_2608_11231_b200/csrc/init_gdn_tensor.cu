@@ -66,7 +66,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
     constexpr int kSHalf = SBF16 ? kSHalfBytes / 2 : kSHalfBytes;   // bytes of half a cached state in the pool's dtype
     __shared__ uint64_t bar_fullT[kStages], bar_freeT[kStages], bar_fullS[2], bar_freeS[2], bar_mma[2], bar_sready;
     __shared__ uint32_t tmem_base;
-    __shared__ int dead;
+    __shared__ volatile int dead;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, r = blockIdx.y;
@@ -192,8 +192,10 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
             }
             mbar_arrive(&bar_freeS[half]);
             if (j == K - 1) {
+                if (!dead) {   // a wait ran out: the status word says so, S0 is left alone
 #pragma unroll
-                for (int i = 0; i < 64; ++i) __stcs(out + static_cast<size_t>(i0 + i) * kD + c, val[i]);
+                    for (int i = 0; i < 64; ++i) __stcs(out + static_cast<size_t>(i0 + i) * kD + c, val[i]);
+                }
             } else {
                 const uint32_t abuf = lane_base + 128 + 128 * (j & 1) + i0;
 #pragma unroll

@@ -38,7 +38,7 @@ init_mamba_exact_stream_kernel(const __grid_constant__ InitArgs a, size_t state_
     unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     __shared__ uint64_t full[kStages], empty[kStages];
     __shared__ float dec[kDecSlots];
-    __shared__ int dead;
+    __shared__ volatile int dead;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -123,6 +123,7 @@ init_mamba_exact_stream_kernel(const __grid_constant__ InitArgs a, size_t state_
                 }
             }
             float *dst = a.S0 + static_cast<size_t>(r) * state_elems + static_cast<size_t>(tile) * kTileElems;
+            if (dead) continue;   // a wait ran out: the status word says so, S0 is left alone
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll

@@ -14,6 +14,13 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline bool dtype_ok(int d) { return d == LKV_DTYPE_F32 || d == LKV_DTYPE_BF16; }
 inline bool compute_ok(int c) { return c == LKV_COMPUTE_AUTO || c == LKV_COMPUTE_FP32 || c == LKV_COMPUTE_TENSOR; }
 
+// Byte ranges [p, p + n) and [q, q + m) share at least one byte (empty or NULL ranges never do).
+inline bool overlaps(const void *p, size_t n, const void *q, size_t m) {
+    if (!p || !q || n == 0 || m == 0) return false;
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p), b = reinterpret_cast<uintptr_t>(q);
+    return a < b + m && b < a + n;
+}
+
 size_t ws_bytes_for(int n_ints, int cap) {
     return kWsHeaderBytes + (n_ints > cap ? align_up(sizeof(int32_t) * static_cast<size_t>(n_ints), 256) : 0);
 }
@@ -27,6 +34,13 @@ int place_indices(IndexBlock<CAP> &blk, const std::vector<int32_t> &ints, void *
         if (!ints.empty()) memcpy(blk.v, ints.data(), sizeof(int32_t) * ints.size());
         return LKV_OK;
     }
+    // The copy reads a host array that dies with this call: a stream capture would record the read, not do it.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    if (cap != cudaStreamCaptureStatusNone) return LKV_ERR_UNSUPPORTED;
     int32_t *dst = reinterpret_cast<int32_t *>(static_cast<char *>(workspace) + kWsHeaderBytes);
     if (cudaMemcpyAsync(dst, ints.data(), sizeof(int32_t) * ints.size(), cudaMemcpyHostToDevice, s) != cudaSuccess) {
         cudaGetLastError();
@@ -75,6 +89,15 @@ int init_impl(const void *states, const void *transitions, const int32_t *chunk_
     if (exact && !transitions) return LKV_ERR_NULL;
     if (!aligned16(S0) || !aligned16(states) || (exact && !aligned16(transitions))) return LKV_ERR_ALIGN;
     const bool pool_bf16 = d->state_dtype == LKV_DTYPE_BF16;
+    {
+        const size_t state_elems = static_cast<size_t>(d->H) * d->d_k * d->d_v;
+        const size_t out_bytes = sizeof(float) * state_elems * n_req;
+        const size_t pool_bytes = (pool_bf16 ? 2 : 4) * state_elems * d->n_chunks;
+        const size_t tr_bytes = sizeof(float) * static_cast<size_t>(d->n_chunks) * d->H *
+                                (d->family == LKV_FAMILY_GDN ? static_cast<size_t>(d->d_k) * d->d_k : 1);
+        if (overlaps(S0, out_bytes, states, total > 0 ? pool_bytes : 0) || (exact && overlaps(S0, out_bytes, transitions, tr_bytes)))
+            return LKV_ERR_OVERLAP;
+    }
     if (d->d_v % (pool_bf16 ? 8 : 4) != 0) return LKV_ERR_UNSUPPORTED;
 
     const int n_ints = (n_req + 1) + (mode == LKV_INIT_INDEX ? n_req : 0) + total;
@@ -192,6 +215,19 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         return LKV_ERR_ALIGN;
     if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
     if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+    {
+        // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
+        const size_t es = d->io_dtype == LKV_DTYPE_BF16 ? 2 : 4, T = static_cast<size_t>(d->T_total);
+        const size_t qk_b = es * T * d->H_k * d->d_k, v_b = es * T * d->H_v * d->d_v, gb_b = sizeof(float) * T * d->H_v;
+        const size_t st_b = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H_v * d->d_k * d->d_v;
+        const void *in[6] = {q, k, v, g, beta, S0};
+        const size_t in_b[6] = {qk_b, qk_b, v ? v_b : 0, gb_b, gb_b, S0 ? st_b : 0};
+        for (int i = 0; i < 6; ++i) {
+            if (overlaps(o, o ? v_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
+            if (!(i == 5 && S_T == S0) && overlaps(S_T, S_T ? st_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
+        }
+        if (overlaps(o, o ? v_b : 0, S_T, S_T ? st_b : 0)) return LKV_ERR_OVERLAP;
+    }
 
     GdnArgs a;
     a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = S_T;
@@ -286,6 +322,19 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
         return LKV_ERR_ALIGN;
     if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
     if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
+    {
+        // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
+        const size_t es = d->io_dtype == LKV_DTYPE_BF16 ? 2 : 4, T = static_cast<size_t>(d->T_total);
+        const size_t x_b = es * T * d->H * d->P, bc_b = es * T * d->G * d->N, dt_b = sizeof(float) * T * d->H;
+        const size_t st_b = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H * d->N * d->P;
+        const void *in[6] = {x, dt, A, B, C, S0};
+        const size_t in_b[6] = {x_b, dt_b, sizeof(float) * d->H, bc_b, bc_b, S0 ? st_b : 0};
+        for (int i = 0; i < 6; ++i) {
+            if (overlaps(y, y ? x_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
+            if (!(i == 5 && S_T == S0) && overlaps(S_T, S_T ? st_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
+        }
+        if (overlaps(y, y ? x_b : 0, S_T, S_T ? st_b : 0)) return LKV_ERR_OVERLAP;
+    }
 
     SsdArgs a;
     a.x = x; a.dt = dt; a.A = A; a.B = B; a.C = C; a.S0 = S0; a.y = y; a.S_T = S_T;
@@ -334,6 +383,14 @@ int lkv_device_status(const void *workspace, void *stream) {
     return word == 0 ? LKV_OK : LKV_ERR_DEVICE_TIMEOUT;
 }
 
+int lkv_selftest_bounded_wait(int poll_limit, void *workspace, void *stream) {
+    if (!workspace) return LKV_ERR_NULL;
+    if (poll_limit < 1 || poll_limit > (1 << 20)) return LKV_ERR_DIM;
+    if (!aligned16(workspace)) return LKV_ERR_ALIGN;
+    return launch_selftest_bounded_wait(static_cast<uint32_t>(poll_limit), static_cast<int32_t *>(workspace),
+                                        static_cast<cudaStream_t>(stream)) == cudaSuccess ? LKV_OK : LKV_ERR_CUDA;
+}
+
 const char *lkv_status_string(int status) {
     switch (status) {
         case LKV_OK: return "ok";
@@ -346,6 +403,7 @@ const char *lkv_status_string(int status) {
         case LKV_ERR_WORKSPACE: return "workspace missing or too small";
         case LKV_ERR_CUDA: return "CUDA runtime call failed";
         case LKV_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case LKV_ERR_OVERLAP: return "an output buffer overlaps an input or another output";
         default: return "unknown status";
     }
 }
@@ -388,6 +446,25 @@ void *static_scratch_for_current_device() {
 }
 }  // namespace
 
+// Status word of the static scratch on the current device: read, and cleared if it was set (nobody else can).
+extern "C" int lkv_device_status_static(void *stream) {
+    void *scratch = static_scratch_for_current_device();
+    if (!scratch) return LKV_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    if (word == 0) return LKV_OK;
+    if (cudaMemsetAsync(scratch, 0, sizeof(word), s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return LKV_ERR_CUDA;
+    }
+    return LKV_ERR_DEVICE_TIMEOUT;
+}
+
 extern "C" int lkv_init_state_batched_static(const void *states, const void *transitions, const int32_t *chunk_ids,
                                              const int32_t *cu_k, int n_req, int mode, const int32_t *sel_index,
                                              void *S0, const lkv_init_desc *d, void *stream) {
@@ -399,11 +476,6 @@ extern "C" int lkv_init_state_batched_static(const void *states, const void *tra
     if (n_ints > LKV_STATIC_MAX_INDEX) return LKV_ERR_WORKSPACE;
     void *scratch = static_scratch_for_current_device();
     if (!scratch) return LKV_ERR_CUDA;
-    // the array keeps the previous call's contents: the status word must start at zero
-    if (cudaMemsetAsync(scratch, 0, kWsHeaderBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
-        cudaGetLastError();
-        return LKV_ERR_CUDA;
-    }
     lkv_init_desc local = *d;
     local.workspace = scratch;
     local.workspace_bytes = LKV_STATIC_SCRATCH_BYTES;

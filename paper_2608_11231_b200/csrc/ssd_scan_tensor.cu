@@ -17,6 +17,8 @@
 // Warps 0-7 epilogue (thread = token row, warpgroup = column half), 8-11 state copy (the only SIMT
 // work on the block-to-block chain), 12-15 per-block scalars and X~ (running ahead of the chain),
 // 16 TMA, 17 MMA issue.  All waits on mbarriers are bounded.
+#include <string.h>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -79,7 +81,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
     unsigned char *sm = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ Bars bars;
     __shared__ uint32_t tmem_base;
-    __shared__ int dead;
+    __shared__ volatile int dead;
     __shared__ float scan_carry[4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -328,7 +330,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 tmem_ld32(lane_base + kTmH + 32 * q, rr);
                 tmem_ld_wait();
                 if (last) {
-                    if (a.S_T) {
+                    if (a.S_T && !dead) {
 #pragma unroll
                         for (int c = 0; c < 32; c += 4)
                             *reinterpret_cast<float4 *>(a.S_T + sbase + static_cast<size_t>(x) * kP + 32 * q + c) =
@@ -453,7 +455,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                     fence_async_smem();
                 } else {
                     const int tok = row0 + t;
-                    if (tok < t_end) {
+                    if (tok < t_end && !dead) {
                         __nv_bfloat16 *dst = y + (static_cast<size_t>(tok) * a.H + h) * kP + 32 * half;
 #pragma unroll
                         for (int c8 = 0; c8 < 4; ++c8)
@@ -481,7 +483,12 @@ cudaError_t launch_ssd_scan_tensor(const SsdArgs &a, cudaStream_t s) {
     CUtensorMap mapX, mapB, mapC, mapY;
     const uint64_t rows = static_cast<uint64_t>(a.T_total);
     const uint64_t x_inner = static_cast<uint64_t>(a.H) * kP, bc_inner = static_cast<uint64_t>(a.G) * kN;
-    if (!make_tensor_map_2d(&mapX, a.x, 2, x_inner, rows, x_inner * 2, 64, kQ, true) ||
+    if (rows == 0) {
+        // no token anywhere: every CTA hands its state through and never touches a tile (and a map of zero rows
+        // cannot be encoded)
+        memset(&mapX, 0, sizeof(mapX));
+        mapB = mapC = mapY = mapX;
+    } else if (!make_tensor_map_2d(&mapX, a.x, 2, x_inner, rows, x_inner * 2, 64, kQ, true) ||
         !make_tensor_map_2d(&mapB, a.B, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
         !make_tensor_map_2d(&mapC, a.C, 2, bc_inner, rows, bc_inner * 2, 64, kQ, true) ||
         (a.y && !make_tensor_map_2d(&mapY, a.y, 2, x_inner, rows, x_inner * 2, 64, kQ, true)))

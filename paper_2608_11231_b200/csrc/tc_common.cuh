@@ -60,9 +60,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
 // Waits for the phase with the given parity.  `dead` is a CTA-wide flag in shared memory: once any
 // wait in the CTA has run out, every later wait returns at once, so a broken pipeline drains in
 // bounded time instead of spinning.  On timeout the device status word is set for the host to read.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *dead, int *status) {
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *dead, int *status, uint32_t limit) {
     if (*dead) return false;
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -80,9 +80,9 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
 }
 // The probe is inline (the common case in a pipeline that runs ahead); the polling loop is one shared
 // function so that the many waits of a warp-specialised kernel do not bloat its instruction footprint.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status, uint32_t limit = kSpinLimit) {
     if (mbar_test_wait(bar, parity)) return true;
-    return mbar_wait_slow(smem_u32(bar), parity, dead, status);
+    return mbar_wait_slow(smem_u32(bar), parity, dead, status, limit);
 }
 
 // ------------------------------------------------------------------ TMA (tiled bulk tensor loads, 2-D)

@@ -36,3 +36,14 @@ def _error_log(request):
     if path and helpers.ERRORS:
         with open(path, "a") as fh:
             fh.write(request.node.nodeid + " " + " ".join(f"{e:.3e}" for e in helpers.ERRORS) + "\n")
+
+
+@pytest.fixture(autouse=True)
+def _device_status_clean(request):
+    """After every GPU test: no kernel of the library gave up a bounded wait on any workspace the binding handed out."""
+    yield
+    if "gpu" not in request.node.keywords:
+        return
+    from paper_2608_11231_b200 import binding as b
+    for ws in list(b._ws_cache.values()):
+        assert b.lkv_device_status(ws) == b.LKV_OK, "a device-side wait timed out during this test"

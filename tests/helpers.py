@@ -25,6 +25,22 @@ def maxrel(x, ref) -> float:
     return err
 
 
+def maxrel_per_head(x, ref, head_axis: int) -> float:
+    """The worst head's own max-norm relative error: max over h of max|x - ref|_h / max|ref|_h.
+
+    A head (or a head of one sequence, with the sequences split by the caller) whose values are small cannot
+    hide behind a large one, as it can in maxrel() over the whole tensor.
+    """
+    x = np.moveaxis(np.asarray(x, dtype=np.float64), head_axis, 0)
+    ref = np.moveaxis(np.asarray(ref, dtype=np.float64), head_axis, 0)
+    worst = 0.0
+    for xh, rh in zip(x, ref):
+        den = np.abs(rh).max()
+        worst = max(worst, float(np.abs(xh).max()) if den == 0.0 else float(np.abs(xh - rh).max() / den))
+    ERRORS.append(worst)
+    return worst
+
+
 def frobrel(x, ref) -> float:
     x = np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)

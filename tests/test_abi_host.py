@@ -13,6 +13,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 FAKE = 0x7F0000000000  # a 16-byte aligned non-NULL "device pointer"; never dereferenced on the host
 
 
+def fake(i):
+    """Distinct fake device buffers, 4 GiB apart (the library checks that outputs do not overlap inputs)."""
+    return FAKE + (i << 32)
+
+
+
 @pytest.fixture(scope="module")
 def lib():
     if not os.path.exists(b.LIB_PATH):
@@ -32,8 +38,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert b.lkv_version() == 100
-    seen = {b.status_string(s) for s in range(0, -10, -1)}
-    assert len(seen) == 10 and "unknown status" not in seen
+    seen = {b.status_string(s) for s in range(0, -11, -1)}
+    assert len(seen) == 11 and "unknown status" not in seen
     assert b.status_string(-99) == "unknown status"
 
 
@@ -44,7 +50,7 @@ def _desc(**kw):
     return b.lkv_init_desc(**base)
 
 
-def _init(lib, d, K=4, mode=b.LKV_INIT_EXACT, states=FAKE, trans=FAKE, S0=FAKE):
+def _init(lib, d, K=4, mode=b.LKV_INIT_EXACT, states=fake(1), trans=fake(2), S0=fake(3)):
     return lib.lkv_init_state(states, trans, K, mode, S0, ctypes.byref(d) if d is not None else None, None)
 
 
@@ -66,8 +72,10 @@ def test_init_state_argument_errors(lib):
     assert _init(lib, _desc(), S0=None) == b.LKV_ERR_NULL
     assert _init(lib, _desc(), states=None) == b.LKV_ERR_NULL
     assert _init(lib, _desc(), trans=None) == b.LKV_ERR_NULL      # exact mode with K >= 2 needs transitions
-    assert _init(lib, _desc(), S0=FAKE + 4) == b.LKV_ERR_ALIGN
-    assert _init(lib, _desc(), states=FAKE + 8) == b.LKV_ERR_ALIGN
+    assert _init(lib, _desc(), S0=fake(3) + 4) == b.LKV_ERR_ALIGN
+    assert _init(lib, _desc(), states=fake(1) + 8) == b.LKV_ERR_ALIGN
+    assert _init(lib, _desc(), S0=fake(1) + 64) == b.LKV_ERR_OVERLAP        # S0 inside the pool of states
+    assert _init(lib, _desc(), S0=fake(2)) == b.LKV_ERR_OVERLAP              # S0 on the transitions
     assert _init(lib, _desc(d_v=6)) == b.LKV_ERR_UNSUPPORTED
     assert _init(lib, _desc(workspace=None)) == b.LKV_ERR_WORKSPACE
     assert _init(lib, _desc(workspace_bytes=16)) == b.LKV_ERR_WORKSPACE
@@ -79,8 +87,8 @@ def test_init_state_batched_argument_errors(lib):
     ids = np.array([0, 1, 2, 3, 1], dtype=np.int32)
     f = lib.lkv_init_state_batched
     call = lambda cu, n, mode=b.LKV_INIT_EXACT, sel=None, idp=ids: f(
-        FAKE, FAKE, idp.ctypes.data if idp is not None else None, cu.ctypes.data if cu is not None else None, n, mode,
-        sel.ctypes.data if sel is not None else None, FAKE, ctypes.byref(d), None)
+        fake(1), fake(2), idp.ctypes.data if idp is not None else None, cu.ctypes.data if cu is not None else None, n, mode,
+        sel.ctypes.data if sel is not None else None, fake(3), ctypes.byref(d), None)
     assert call(None, 2) == b.LKV_ERR_NULL
     assert call(np.array([1, 3, 5], dtype=np.int32), 2) == b.LKV_ERR_INDEX      # must start at 0
     assert call(np.array([0, 4, 3], dtype=np.int32), 2) == b.LKV_ERR_INDEX      # not monotone
@@ -100,8 +108,8 @@ def _gdn_desc(**kw):
 
 
 def test_gdn_fwd_argument_errors(lib):
-    f = lambda d, q=FAKE, o=FAKE, S0=None: lib.lkv_gdn_fwd(q, FAKE, FAKE, FAKE, FAKE, S0, o, None,
-                                                           ctypes.byref(d) if d is not None else None, None)
+    f = lambda d, q=fake(1), o=fake(7), S0=None, S_T=None: lib.lkv_gdn_fwd(q, fake(2), fake(3), fake(4), fake(5), S0, o, S_T,
+                                                                            ctypes.byref(d) if d is not None else None, None)
     assert f(None) == b.LKV_ERR_NULL
     assert f(_gdn_desc(io_dtype=4)) == b.LKV_ERR_MODE
     assert f(_gdn_desc(H_v=3)) == b.LKV_ERR_DIM
@@ -113,8 +121,12 @@ def test_gdn_fwd_argument_errors(lib):
     cu = np.array([0, 120, 100], dtype=np.int32)
     assert f(_gdn_desc(n_seq=2, cu_seqlens=cu.ctypes.data)) == b.LKV_ERR_INDEX
     assert f(_gdn_desc(), q=None) == b.LKV_ERR_NULL
-    assert f(_gdn_desc(), o=FAKE + 2) == b.LKV_ERR_ALIGN
-    assert f(_gdn_desc(), S0=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(), o=fake(7) + 2) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(), S0=fake(6) + 4) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(), o=fake(3)) == b.LKV_ERR_OVERLAP                  # o on v
+    assert f(_gdn_desc(), o=fake(1) + 1024) == b.LKV_ERR_OVERLAP           # o inside q
+    assert f(_gdn_desc(), S0=fake(6), S_T=fake(6) + 256) == b.LKV_ERR_OVERLAP   # S_T may be S0 itself, not a shifted view
+    assert f(_gdn_desc(), S_T=fake(4)) == b.LKV_ERR_OVERLAP                # S_T on g
     assert f(_gdn_desc(d_v=48)) == b.LKV_ERR_UNSUPPORTED
     assert f(_gdn_desc(workspace=None)) == b.LKV_ERR_WORKSPACE
     assert f(_gdn_desc(compute=b.LKV_COMPUTE_TENSOR, d_k=24, d_v=32)) == b.LKV_ERR_UNSUPPORTED
@@ -129,27 +141,29 @@ def _ssd_desc(**kw):
 
 
 def test_ssd_fwd_argument_errors(lib):
-    f = lambda d, x=FAKE, A=FAKE, y=FAKE: lib.lkv_ssd_fwd(x, FAKE, A, FAKE, FAKE, None, y, None,
-                                                          ctypes.byref(d) if d is not None else None, None)
+    f = lambda d, x=fake(1), A=fake(3), y=fake(7): lib.lkv_ssd_fwd(x, fake(2), A, fake(4), fake(5), None, y, None,
+                                                                   ctypes.byref(d) if d is not None else None, None)
     assert f(None) == b.LKV_ERR_NULL
     assert f(_ssd_desc(compute=-1)) == b.LKV_ERR_MODE
     assert f(_ssd_desc(G=3)) == b.LKV_ERR_DIM
     assert f(_ssd_desc(N=0)) == b.LKV_ERR_DIM
     assert f(_ssd_desc(), A=None) == b.LKV_ERR_NULL
     assert f(_ssd_desc(), x=None) == b.LKV_ERR_NULL
-    assert f(_ssd_desc(), y=FAKE + 8) == b.LKV_ERR_ALIGN
+    assert f(_ssd_desc(), y=fake(7) + 8) == b.LKV_ERR_ALIGN
+    assert f(_ssd_desc(), y=fake(1)) == b.LKV_ERR_OVERLAP                  # y on x
+    assert f(_ssd_desc(), y=fake(5) + 32) == b.LKV_ERR_OVERLAP             # y inside C
     assert f(_ssd_desc(P=48)) == b.LKV_ERR_UNSUPPORTED
     assert f(_ssd_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE
 
 
 def test_artifact_producers_argument_errors(lib):
-    t = lambda d, k=FAKE, out=FAKE: lib.lkv_gdn_chunk_transition(k, FAKE, FAKE, out,
+    t = lambda d, k=fake(1), out=fake(7): lib.lkv_gdn_chunk_transition(k, fake(2), fake(3), out,
                                                                   ctypes.byref(d) if d is not None else None, None)
     assert t(None) == b.LKV_ERR_NULL
     assert t(_gdn_desc(d_k=128, d_v=64)) == b.LKV_ERR_DIM             # the transition is d_k x d_k: d_v must equal d_k
     assert t(_gdn_desc(), out=None) == b.LKV_ERR_NULL
     assert t(_gdn_desc(), k=None) == b.LKV_ERR_NULL
-    assert t(_gdn_desc(), out=FAKE + 4) == b.LKV_ERR_ALIGN
+    assert t(_gdn_desc(), out=fake(7) + 4) == b.LKV_ERR_ALIGN
     assert t(_gdn_desc(workspace=None)) == b.LKV_ERR_WORKSPACE
     m = lambda d, dt=FAKE, A=FAKE, out=FAKE: lib.lkv_mamba_chunk_logdecay(dt, A, out,
                                                                           ctypes.byref(d) if d is not None else None, None)
@@ -160,9 +174,9 @@ def test_artifact_producers_argument_errors(lib):
     assert m(_ssd_desc(), dt=FAKE + 4) == b.LKV_ERR_ALIGN
     assert m(_ssd_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE
     # final-state-only scans: o / y may be NULL, but not together with S_T
-    g = lib.lkv_gdn_fwd(FAKE, FAKE, FAKE, FAKE, FAKE, None, None, None, ctypes.byref(_gdn_desc()), None)
+    g = lib.lkv_gdn_fwd(fake(1), fake(2), fake(3), fake(4), fake(5), None, None, None, ctypes.byref(_gdn_desc()), None)
     assert g == b.LKV_ERR_NULL
-    y = lib.lkv_ssd_fwd(FAKE, FAKE, FAKE, FAKE, FAKE, None, None, None, ctypes.byref(_ssd_desc()), None)
+    y = lib.lkv_ssd_fwd(fake(1), fake(2), fake(3), fake(4), fake(5), None, None, None, ctypes.byref(_ssd_desc()), None)
     assert y == b.LKV_ERR_NULL
 
 
@@ -198,3 +212,10 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(b, "LIB_PATH", str(tmp_path / "liblkv.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         b.load()
+
+
+def test_selftest_and_static_status_argument_errors(lib):
+    assert lib.lkv_selftest_bounded_wait(1000, None, None) == b.LKV_ERR_NULL
+    assert lib.lkv_selftest_bounded_wait(0, FAKE, None) == b.LKV_ERR_DIM
+    assert lib.lkv_selftest_bounded_wait(1 << 21, FAKE, None) == b.LKV_ERR_DIM
+    assert lib.lkv_selftest_bounded_wait(1000, FAKE + 4, None) == b.LKV_ERR_ALIGN

@@ -58,3 +58,36 @@ def test_static_scratch_rejects_oversized_requests():
         b.lkv_init_state_batched_static(pool, lam, big_ids, big_cu, n_req, b.LKV_INIT_EXACT, None,
                                         family=b.LKV_FAMILY_MAMBA2)
     assert e.value.status == b.LKV_ERR_WORKSPACE
+
+
+def test_static_scratch_gdn_exact_on_the_tensor_cores_and_its_status_word():
+    """The kernel with bounded device waits (GDN composition, d = 128) on the library's own scratch:
+    index list in the scratch array, results equal to the workspace entry point, status word clean."""
+    import torch
+    rng = np.random.default_rng(5)
+    n, H, d = 16, 2, 128
+    pool = torch.from_numpy(wl.synthetic_states(rng, n, H, d, d)).cuda()
+    tr = torch.from_numpy(wl.synthetic_gdn_transitions(rng, n, H, d)).cuda()
+    n_req, K = 140, 30
+    ids = rng.integers(0, n, size=n_req * K).astype(np.int32)
+    cu = (np.arange(n_req + 1) * K).astype(np.int32)
+    assert 2 * n_req + 1 + ids.size > 4000
+    out = torch.full((n_req, H, d, d), float("nan"), device="cuda")
+    assert b.lkv_device_status_static() == b.LKV_OK
+    for compute in (b.LKV_COMPUTE_TENSOR, b.LKV_COMPUTE_FP32):
+        ref = b.lkv_init_state_batched(pool, tr, ids, cu, n_req, b.LKV_INIT_EXACT, None, family=b.LKV_FAMILY_GDN,
+                                       compute=compute)
+        got = b.lkv_init_state_batched_static(pool, tr, ids, cu, n_req, b.LKV_INIT_EXACT, None, out,
+                                              family=b.LKV_FAMILY_GDN, compute=compute)
+        torch.cuda.synchronize()
+        assert torch.equal(got, ref), compute
+        assert b.lkv_device_status_static() == b.LKV_OK
+    # an argument error is found before anything reaches the stream: the earlier result stays as it was
+    keep = out.clone()
+    with pytest.raises(b.LkvError) as e:
+        bad = ids.copy()
+        bad[7] = n                                           # chunk id out of range
+        b.lkv_init_state_batched_static(pool, tr, bad, cu, n_req, b.LKV_INIT_EXACT, None, out, family=b.LKV_FAMILY_GDN)
+    assert e.value.status == b.LKV_ERR_INDEX
+    torch.cuda.synchronize()
+    assert torch.equal(out, keep) and b.lkv_device_status_static() == b.LKV_OK
