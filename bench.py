@@ -130,8 +130,26 @@ class Family:
         self.ws_scan = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
         self.d2h_bytes = self.host_out.numel() * 2 + self.host_S_T.numel() * 4
-        self.pool_bytes_unique = h["states"].numel() * 4 + h["trans"].numel() * 4
+        # bytes an exact composition must move at least once: every pool state and transition that some request reads
+        # (a request's first chunk contributes its state only: its transition multiplies nothing), plus S0 written
+        first = set(int(self.ids[self.cu_k[r]]) for r in range(self.n_req) if ks[r] > 0)
+        later = set(int(i) for r in range(self.n_req) for i in self.ids[self.cu_k[r] + 1:self.cu_k[r + 1]])
+        per_state = int(np.prod(self.state_shape)) * 4
+        per_trans = h["trans"][0].numel() * 4
+        self.compose_bytes = len(first | later) * per_state + len(later) * per_trans + self.n_req * per_state
+        self.set_bytes = self.h2d_bytes
         self.launches = 3
+
+    def cold_copy(self):
+        """A second instance over the same host data with device buffers of its own (inputs and outputs): launches
+        that rotate over several of them find none of their inputs in L2."""
+        import copy
+        c = copy.copy(self)
+        c.dev = {n: t.clone() for n, t in self.dev.items()}
+        for n in ("S0_last", "S0", "S_T", "out"):
+            setattr(c, n, getattr(self, n).clone())
+        c.ws_init, c.ws_scan = self.ws_init.clone(), self.ws_scan.clone()
+        return c
 
     def upload(self):
         for n, t in self.host.items():
@@ -286,53 +304,32 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+L2_BYTES = 126e6
+SMALL_KERNEL_US = 100.0   # below this a single launch between two events is dominated by the 2.048 us event resolution
+                          # (on these boxes) and the launch gap: such kernels are timed many launches at a time instead
 
-    from paper_2608_11231_b200 import binding as b
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    b.load()
+class Timer:
+    """Device timing helpers of one rank (CUDA events on the current stream, max over ranks)."""
 
-    reqs = build_requests(args.workload, rank)
-    fams = []
-    for fam in ("mamba2", "gdn"):
-        sub = [r for r in reqs if r["family"] == fam]
-        if sub:
-            fams.append(Family(fam, sub, seed=100 + rank * 10 + len(fams), torch=torch, b=b))
-    torch.cuda.synchronize()
-    context_tokens = sum(f.context_tokens for f in fams)
-    scan_tokens = sum(f.scan_tokens for f in fams)
-    job_context_tokens = context_tokens
-    job_scan_tokens = scan_tokens
+    def __init__(self, torch, dist, world):
+        from paper_2608_11231_b200 import sharding
+        self.torch, self.dist, self.world, self.sharding = torch, dist, world, sharding
+        self.flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
 
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.world > 1:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
 
-    from paper_2608_11231_b200 import sharding
+    def max_over_ranks(self, x: float) -> float:
+        return self.sharding.job_step_ms(x, self.dist if self.world > 1 else None, "cuda")
 
-    def max_over_ranks(x: float) -> float:
-        return sharding.job_step_ms(x, dist if world > 1 else None, "cuda")
-
-    total_input_bytes = sum(f.h2d_bytes for f in fams)
-    cold_by_size = total_input_bytes > 4 * 126e6        # inputs far larger than the 126 MB L2
-    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
-
-    def flush_l2():
-        flush_buf.zero_()
-
-    def graph_of(fn):
+    def graph_of(self, fn):
         """Capture fn (launches only, no allocation) into a CUDA graph so that host overhead of the
         Python binding does not enter device timings of microsecond-scale kernels."""
+        torch = self.torch
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -344,94 +341,200 @@ def run_ours(args):
             fn()
         return g
 
-    def timed_back_to_back(replay, steps):
+    def back_to_back(self, replay, steps):
+        torch = self.torch
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
+        self.barrier()
         ev0.record()
         for _ in range(steps):
             replay()
         ev1.record()
-        barrier()
-        return max_over_ranks(ev0.elapsed_time(ev1) / steps)  # ms per step
+        self.barrier()
+        return self.max_over_ranks(ev0.elapsed_time(ev1) / steps)  # ms per step
 
-    def timed_flushed(replay, steps, reduce="mean"):
-        """Each iteration timed alone, L2 flushed (untimed) before it."""
+    def flushed(self, replay, steps):
+        """Each iteration timed alone, L2 flushed (untimed) before it.  Returns the list of ms."""
+        torch = self.torch
         ts = []
-        barrier()
+        self.barrier()
         for _ in range(steps):
-            flush_l2()
+            self.flush_buf.zero_()
             ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             ev0.record()
             replay()
             ev1.record()
             ev1.synchronize()
             ts.append(ev0.elapsed_time(ev1))
-        barrier()
-        t = statistics.median(ts) if reduce == "median" else sum(ts) / len(ts)
-        return max_over_ranks(t)
+        self.barrier()
+        return ts
+
+    def kernel_us(self, fns, set_bytes, steps):
+        """Device time of one launch of a kernel, cold inputs.  fns: the same call over several sets of buffers.
+
+        A launch longer than SMALL_KERNEL_US is timed alone between two events after an L2 flush (median, p90 over
+        `steps`).  A shorter one is timed R launches at a time inside one graph between one event pair, the launches
+        rotating over n sets of buffers whose total size exceeds L2 (so every launch finds its inputs in HBM), and the
+        time divided by R; median and p90 over 9 such replays."""
+        g = self.graph_of(fns[0])
+        ts = sorted(1e3 * t for t in self.flushed(g.replay, steps))
+        single = dict(us=statistics.median(ts), p90_us=ts[min(len(ts) - 1, int(0.9 * len(ts)))],
+                      method="one launch per event pair, L2 flushed before it")
+        if single["us"] >= SMALL_KERNEL_US or len(fns) < 2:
+            return single
+        n = len(fns)
+        R = max(24, n)
+
+        def many():
+            for i in range(R):
+                fns[i % n]()
+        gm = self.graph_of(many)
+        per = []
+        for _ in range(9):
+            t = self.flushed(gm.replay, 1)[0]
+            per.append(1e3 * t / R)
+        per.sort()
+        return dict(us=statistics.median(per), p90_us=per[min(len(per) - 1, int(0.9 * len(per)))],
+                    method=f"{R} launches per event pair rotating over {n} buffer sets "
+                           f"({n * set_bytes / 1e6:.0f} MB in total, L2 is 126 MB), time / {R}",
+                    one_launch_flushed_us=single["us"], event_resolution_us=2.048)
+
+
+def n_cold_sets(set_bytes: float) -> int:
+    """Buffer sets needed for their total to exceed L2 with margin: at least 4, at most 48."""
+    return int(min(48, max(4, -(-1.5 * L2_BYTES // max(set_bytes, 1.0)))))
+
+
+def host_us_per_call(fn, torch, calls=50):
+    """Host time of one call of the Python binding + C entry point (argument checks, tensor maps, launch), measured
+    while the stream is kept short of work: what a caller pays on its own thread per launch."""
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        fn()
+    dt = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    return 1e6 * dt / calls
+
+
+def measure_workload(name, rank, world, args, torch, b, dist, timer, peaks, with_e2e=True):
+    """All device timings of one workload on this rank: whole step, every kernel alone, the full-prefill reference."""
+    reqs = build_requests(name, rank)
+    fams = []
+    for fam in ("mamba2", "gdn"):
+        sub = [r for r in reqs if r["family"] == fam]
+        if sub:
+            fams.append(Family(fam, sub, seed=100 + rank * 10 + len(fams), torch=torch, b=b))
+    torch.cuda.synchronize()
+    context_tokens = sum(f.context_tokens for f in fams)
+    scan_tokens = sum(f.scan_tokens for f in fams)
+    total_input_bytes = sum(f.h2d_bytes for f in fams)
+    cold_by_size = total_input_bytes > 4 * L2_BYTES        # inputs far larger than the 126 MB L2
+    steps = args.steps
 
     def step():
         for f in fams:
             f.step()
 
-    e2e_streams = [torch.cuda.Stream() for _ in fams]
-
-    def step_e2e():
-        # one stream per family: the device->host copies of one overlap the host->device copies of the other
-        cur = torch.cuda.current_stream()
-        for f, st in zip(fams, e2e_streams):
-            st.wait_stream(cur)
-            with torch.cuda.stream(st):
-                f.upload()
-                f.step()
-                f.download()
-        for st in e2e_streams:
-            cur.wait_stream(st)
-
-    # clocks are sampled from the warm-up to the end of the end-to-end steps: the GPU is busy throughout
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
-    g_step = graph_of(step)
+    g_step = timer.graph_of(step)
     for _ in range(max(args.warmup, 3)):
         g_step.replay()
     if cold_by_size:
-        ms = timed_back_to_back(g_step.replay, args.steps)
+        ms = timer.back_to_back(g_step.replay, steps)
     else:
-        ms = timed_flushed(g_step.replay, args.steps)
-    # per-kernel device times: each kernel alone in its own graph, L2 flushed before every launch, median
+        ts = timer.flushed(g_step.replay, steps)
+        ms = timer.max_over_ranks(sum(ts) / len(ts))
+
+    # per-kernel device times, each kernel alone
     parts = {}
     for f in fams:
-        for name, fn in (("init_last", f.init_last), ("init_exact", f.init_exact), ("scan", f.scan)):
-            g = graph_of(fn)
-            parts[f"{f.fam}.{name}"] = timed_flushed(g.replay, max(args.steps, 5), reduce="median")
-    e2e_steps = max(1, min(args.steps, 3))
-    step_e2e()
-    ms_e2e = timed_back_to_back(step_e2e, e2e_steps)
+        sets = [f]
+        if not cold_by_size:
+            sets += [f.cold_copy() for _ in range(n_cold_sets(f.set_bytes) - 1)]
+        for kname in ("init_last", "init_exact", "scan"):
+            r = timer.kernel_us([getattr(x, kname) for x in sets], f.set_bytes, max(steps, 7))
+            r["us"] = 1e3 * timer.max_over_ranks(1e-3 * r["us"])
+            parts[f"{f.fam}.{kname}"] = r
+        del sets
+    host_us = {}
+    if rank == 0:
+        for f in fams:
+            host_us[f"{f.fam}.init_exact"] = host_us_per_call(f.init_exact, torch)
+            host_us[f"{f.fam}.scan"] = host_us_per_call(f.scan, torch, calls=20)
+
+    ms_e2e, e2e_steps = None, 0
+    if with_e2e:
+        e2e_streams = [torch.cuda.Stream() for _ in fams]
+
+        def step_e2e():
+            # one stream per family: the device->host copies of one overlap the host->device copies of the other
+            cur = torch.cuda.current_stream()
+            for f, st in zip(fams, e2e_streams):
+                st.wait_stream(cur)
+                with torch.cuda.stream(st):
+                    f.upload()
+                    f.step()
+                    f.download()
+            for st in e2e_streams:
+                cur.wait_stream(st)
+        e2e_steps = max(1, min(steps, 3))
+        step_e2e()
+        ms_e2e = timer.back_to_back(step_e2e, e2e_steps)
+
     # full-prefill reference (single-family configurations): one request's whole context scanned from the empty state
     full = {}
-    if args.workload in ("cfg1", "cfg2", "cfg3"):
+    if name in ("cfg1", "cfg2", "cfg3"):
         for f in fams:
             f.make_full_prefill(f.reqs[0]["total"])
-            g = graph_of(f.full_prefill)
-            t = timed_flushed(g.replay, max(args.steps, 5), reduce="median")
+            g = timer.graph_of(f.full_prefill)
+            t = 1e-3 * statistics.median(1e3 * x for x in timer.flushed(g.replay, max(steps, 5)))
             # the same request served from the cache: its share of the batched init calls plus its recompute scan
-            t_cached = (parts[f"{f.fam}.init_exact"] + parts[f"{f.fam}.scan"]) / f.n_req
+            t_cached = 1e-3 * (parts[f"{f.fam}.init_exact"]["us"] + parts[f"{f.fam}.scan"]["us"]) / f.n_req
             full[f.fam] = dict(tokens=f.full_tokens, us=1e3 * t, tokens_per_s=f.full_tokens / (t * 1e-3),
                                cached_path_us_per_request=1e3 * t_cached, cached_over_full=t_cached / t)
-    clocks = sampler.stop() if rank == 0 else None
+            del f.full, f.full_out
 
+    detail = {}
+    for f in fams:
+        us = {k: parts[f"{f.fam}.{k}"]["us"] for k in ("init_last", "init_exact", "scan")}
+        flops = gdn_scan_flops(f.scan_tokens) if f.fam == "gdn" else ssd_scan_flops(f.scan_tokens)
+        tf = flops / (us["scan"] * 1e-6) / 1e12
+        tpeak = peaks["bf16_tflops_sustained"] if us["scan"] > 50e3 else peaks["bf16_tflops"]
+        gbs = f.compose_bytes / (us["init_exact"] * 1e-6) / 1e9
+        detail[f.fam] = dict(
+            requests=f.n_req, context_tokens=f.context_tokens, scan_tokens=f.scan_tokens,
+            init_last_us=us["init_last"], init_exact_us=us["init_exact"], scan_us=us["scan"],
+            init_exact_p90_us=parts[f"{f.fam}.init_exact"]["p90_us"], scan_p90_us=parts[f"{f.fam}.scan"]["p90_us"],
+            timing={k: parts[f"{f.fam}.{k}"]["method"] for k in ("init_exact", "scan")},
+            scan_tokens_per_s=f.scan_tokens / (us["scan"] * 1e-6), scan_tflops=tf, scan_frac_of_tensor_peak=tf / tpeak,
+            compose_bytes=f.compose_bytes, compose_gbs=gbs, compose_frac_of_hbm=gbs / peaks["hbm_gbs"])
+        if host_us:
+            detail[f.fam]["host_us_per_call"] = dict(init_exact=round(host_us[f"{f.fam}.init_exact"], 1),
+                                                     scan=round(host_us[f"{f.fam}.scan"], 1))
+    return dict(name=name, reqs=reqs, fams=fams, ms=ms, ms_e2e=ms_e2e, e2e_steps=e2e_steps, parts=parts, full=full,
+                detail=detail, context_tokens=context_tokens, scan_tokens=scan_tokens, cold_by_size=cold_by_size)
+
+
+def l2_note(cold_by_size):
+    return ("inputs far larger than L2, steps timed back to back" if cold_by_size else
+            "L2 flushed (512 MiB write, untimed) before every timed step")
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_11231_b200 import binding as b
+    from paper_2608_11231_b200 import sharding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
     if world > 1:
-        job_context_tokens = sharding.job_total(context_tokens, dist, "cuda")
-        job_scan_tokens = sharding.job_total(scan_tokens, dist, "cuda")
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    peaks = {}
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    b.load()
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
             peaks = json.load(fh)
@@ -439,38 +542,60 @@ def run_ours(args):
     except OSError:
         peaks = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
         peak_src = "fallback"
+    timer = Timer(torch, dist, world)
 
-    # dominant kernel: the scan of the family with the larger share of the step
-    dom = max(parts, key=parts.get)
+    # clocks are sampled from the warm-up to the end of the end-to-end steps: the GPU is busy throughout
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    m = measure_workload(args.workload, rank, world, args, torch, b, dist, timer, peaks)
+    clocks = sampler.stop() if rank == 0 else None
+    ms, ms_e2e, parts, fams = m["ms"], m["ms_e2e"], m["parts"], m["fams"]
+    job_context_tokens, job_scan_tokens = m["context_tokens"], m["scan_tokens"]
+    if world > 1:
+        job_context_tokens = sharding.job_total(m["context_tokens"], dist, "cuda")
+        job_scan_tokens = sharding.job_total(m["scan_tokens"], dist, "cuda")
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # dominant kernel: the one with the largest share of the step
+    dom = max(parts, key=lambda k: parts[k]["us"])
     fam_name, kern = dom.split(".")
     f = next(x for x in fams if x.fam == fam_name)
+    dom_ms = 1e-3 * parts[dom]["us"]
     if kern == "scan":
         flops = gdn_scan_flops(f.scan_tokens) if fam_name == "gdn" else ssd_scan_flops(f.scan_tokens)
-        achieved = flops / (parts[dom] * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained"] if parts[dom] > 50.0 else peaks["bf16_tflops"]
+        achieved = flops / (dom_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained"] if dom_ms > 50.0 else peaks["bf16_tflops"]
         per_token = NCU_DRAM_BYTES_PER_TOKEN.get(dom)
         roof = dict(bound="tensor", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak,
                     traffic=None if per_token is None else per_token * f.scan_tokens,
                     traffic_source="ncu dram bytes of a smaller launch of the same kernel, scaled by tokens", kernel=dom,
                     peak_source=peak_src)
     else:
-        nbytes = f.pool_bytes_unique + f.S0.numel() * 4
-        achieved = nbytes / (parts[dom] * 1e-3) / 1e9
+        achieved = f.compose_bytes / (dom_ms * 1e-3) / 1e9
         roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                     frac=achieved / peaks["hbm_gbs"], traffic=None, kernel=dom, peak_source=peak_src)
 
-    detail = {}
-    for f in fams:
-        t_scan = parts[f"{f.fam}.scan"] * 1e-3
-        flops = gdn_scan_flops(f.scan_tokens) if f.fam == "gdn" else ssd_scan_flops(f.scan_tokens)
-        comp_bytes = f.pool_bytes_unique + f.S0.numel() * 4
-        detail[f.fam] = dict(
-            requests=f.n_req, context_tokens=f.context_tokens, scan_tokens=f.scan_tokens,
-            init_last_us=1e3 * parts[f"{f.fam}.init_last"], init_exact_us=1e3 * parts[f"{f.fam}.init_exact"],
-            scan_us=1e3 * parts[f"{f.fam}.scan"], scan_tokens_per_s=f.scan_tokens / t_scan,
-            scan_tflops=flops / t_scan / 1e12,
-            compose_gbs_unique=comp_bytes / (parts[f"{f.fam}.init_exact"] * 1e-3) / 1e9,
-            compose_frac_of_hbm=comp_bytes / (parts[f"{f.fam}.init_exact"] * 1e-3) / 1e9 / peaks["hbm_gbs"])
+    RUN = dict(requests=len(m["reqs"]), context_tokens=m["context_tokens"], scan_tokens=m["scan_tokens"],
+               cold_by_size=m["cold_by_size"], h2d=sum(x.h2d_bytes for x in fams), d2h=sum(x.d2h_bytes for x in fams),
+               e2e_steps=m["e2e_steps"], launches=sum(x.launches for x in fams), detail=m["detail"], full=m["full"])
+
+    # the other single-GPU configurations, same protocol (a one-GPU run of the default workload only)
+    configs = {}
+    if world == 1 and args.workload == "cfg4" and not args.no_configs:
+        del m, fams, f
+        torch.cuda.empty_cache()
+        for name in ("cfg1", "cfg2", "cfg3"):
+            c = measure_workload(name, 0, 1, args, torch, b, dist, timer, peaks, with_e2e=False)
+            configs[name] = dict(ms_per_step=c["ms"], value=c["context_tokens"] / (c["ms"] * 1e-3), unit=UNIT,
+                                 requests=len(c["reqs"]), context_tokens=c["context_tokens"],
+                                 scan_tokens=c["scan_tokens"], l2=l2_note(c["cold_by_size"]), kernels=c["detail"],
+                                 full_prefill=c["full"])
+            del c
+            torch.cuda.empty_cache()
 
     base, _ = cpu_baseline_sample() if world == 1 else (None, None)
     if base is not None:
@@ -487,18 +612,19 @@ def run_ours(args):
         metric=METRIC, value=job_context_tokens / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
         warmup=max(args.warmup, 3), ms_per_step=ms, higher_is_better=True, scaling="weak", vs_baseline=None,
         dtype="bf16", data="synthetic",
-        config=dict(workload=args.workload, requests=len(reqs), context_tokens=context_tokens,
-                    scan_tokens=scan_tokens, l2="inputs far larger than L2, steps timed back to back" if cold_by_size else
-                    "L2 flushed (512 MiB write, untimed) before every timed step", timing="CUDA-graph replay, CUDA events",
-                    sharding="requests across ranks, no collective"),
+        config=dict(workload=args.workload, requests=RUN["requests"], context_tokens=RUN["context_tokens"],
+                    scan_tokens=RUN["scan_tokens"], l2=l2_note(RUN["cold_by_size"]),
+                    timing="CUDA-graph replay, CUDA events", sharding="requests across ranks, no collective"),
         e2e=dict(value=job_context_tokens / (ms_e2e * 1e-3), unit=UNIT,
-                 h2d_bytes_per_step=sum(f.h2d_bytes for f in fams), d2h_bytes_per_step=sum(f.d2h_bytes for f in fams),
-                 ms_per_step=ms_e2e, steps=e2e_steps),
-        gpu_launches=sum(f.launches for f in fams) * args.steps,
+                 h2d_bytes_per_step=RUN["h2d"], d2h_bytes_per_step=RUN["d2h"],
+                 ms_per_step=ms_e2e, steps=RUN["e2e_steps"]),
+        gpu_launches=RUN["launches"] * args.steps,
         scan_tokens_per_s=job_scan_tokens / (ms * 1e-3),
-        roofline=roof, kernels=detail, clocks=clocks)
-    if full:
-        line["full_prefill"] = full
+        roofline=roof, kernels=RUN["detail"], clocks=clocks)
+    if RUN["full"]:
+        line["full_prefill"] = RUN["full"]
+    if configs:
+        line["configs"] = configs
     if base is not None:
         line["cpu_baseline"] = base
     print(json.dumps(line))
@@ -508,7 +634,7 @@ def run_ours(args):
 
 def run_sweep(args):
     """--sweep: microseconds per exact composition against K, both families, batch 1 and batch 8 (every request
-    with its own pool entries), L2 flushed before every timed launch.  Prints one JSON line of its own."""
+    with its own pool entries), cold inputs (Timer.kernel_us).  Prints one JSON line of its own."""
     import torch
 
     from paper_2608_11231_b200 import binding as b
@@ -519,7 +645,7 @@ def run_sweep(args):
             hbm = json.load(fh)["hbm_gbs"]
     except OSError:
         hbm = 6650.0
-    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    timer = Timer(torch, None, 1)
     gen = torch.Generator(device="cuda").manual_seed(7)
     rows = []
     for fam in ("mamba2", "gdn"):
@@ -530,44 +656,36 @@ def run_sweep(args):
         for n_req in (1, 8):
             for K in (1, 2, 4, 8, 16, 32, 64):
                 n_pool = n_req * K
-                states = torch.randn((n_pool, H, dk, dv), generator=gen, device="cuda")
-                if fam == "gdn":
-                    trans = torch.randn((n_pool, H, dk, dk), generator=gen, device="cuda") * (0.45 / dk ** 0.5)
-                else:
-                    trans = -2.0 * torch.rand((n_pool, H), generator=gen, device="cuda")
                 ids = np.arange(n_pool, dtype=np.int32)
                 cu_k = (np.arange(n_req + 1) * K).astype(np.int32)
-                S0 = torch.empty((n_req, H, dk, dv), device="cuda")
-                ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
-
-                def fn():
-                    b.lkv_init_state_batched(states, trans, ids, cu_k, n_req, b.LKV_INIT_EXACT, None, S0,
-                                             family=code, workspace_t=ws)
-                for _ in range(3):
-                    fn()
-                torch.cuda.synchronize()
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g):
-                    fn()
-                ts = []
-                for _ in range(max(args.steps, 7)):
-                    flush_buf.zero_()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    g.replay()
-                    e1.record()
-                    e1.synchronize()
-                    ts.append(e0.elapsed_time(e1) * 1e3)
-                us = statistics.median(ts)
-                p90 = sorted(ts)[min(len(ts) - 1, int(0.9 * len(ts)))]
-                nbytes = (states.numel() + S0.numel()) * 4 + trans.numel() * 4
+                tr_bytes = n_pool * H * (dk * dk if fam == "gdn" else 1) * 4
+                set_bytes = (n_pool + n_req) * H * dk * dv * 4 + tr_bytes
+                fns, keep = [], []
+                for _ in range(n_cold_sets(set_bytes)):
+                    states = torch.randn((n_pool, H, dk, dv), generator=gen, device="cuda")
+                    if fam == "gdn":
+                        trans = torch.randn((n_pool, H, dk, dk), generator=gen, device="cuda") * (0.45 / dk ** 0.5)
+                    else:
+                        trans = -2.0 * torch.rand((n_pool, H), generator=gen, device="cuda")
+                    S0 = torch.empty((n_req, H, dk, dv), device="cuda")
+                    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+                    keep.append((states, trans, S0, ws))
+                    fns.append(lambda t=keep[-1]: b.lkv_init_state_batched(t[0], t[1], ids, cu_k, n_req, b.LKV_INIT_EXACT,
+                                                                           None, t[2], family=code, workspace_t=t[3]))
+                r = timer.kernel_us(fns, set_bytes, max(args.steps, 7))
+                nbytes = set_bytes
                 if fam == "gdn":   # the first chunk's transition is never read
                     nbytes -= n_req * H * dk * dk * 4
-                rows.append(dict(family=fam, requests=n_req, K=K, us=round(us, 2), p90_us=round(p90, 2), gbs=round(nbytes / us / 1e3, 1),
-                                 frac_of_hbm=round(nbytes / us / 1e3 / hbm, 3)))
-                del states, trans, S0
-    print(json.dumps(dict(sweep="compose_us_vs_K", timing="graph replay of one launch between CUDA events (includes "
-                          "about 2 us of launch gap), L2 flushed before each, median", rows=rows)))
+                rows.append(dict(family=fam, requests=n_req, K=K, us=round(r["us"], 2), p90_us=round(r["p90_us"], 2),
+                                 gbs=round(nbytes / r["us"] / 1e3, 1), frac_of_hbm=round(nbytes / r["us"] / 1e3 / hbm, 3),
+                                 launches_per_event_pair=1 if "one launch" in r["method"] else max(24, len(fns)),
+                                 buffer_sets=len(fns)))
+                del fns, keep
+                torch.cuda.empty_cache()
+    print(json.dumps(dict(sweep="compose_us_vs_K", timing="kernels under 100 us: 24 or more launches per CUDA-event pair "
+                          "inside one graph, rotating over buffer sets whose total exceeds L2, time divided by the "
+                          "launches, median and p90 of 9 replays; longer ones: one launch per event pair after an L2 "
+                          "flush, median and p90", rows=rows)))
 
 
 def run_artifacts(args):
@@ -626,6 +744,38 @@ def run_artifacts(args):
                           "inputs (about 1.1 GB per family) larger than L2, median", calls=out)))
 
 
+def run_dry(args):
+    """--dry-run: every rank on CPU (gloo); the step is a stand-in that sleeps (rank + 1) ms.  Same request sharding,
+    same max-over-ranks time and whole-job token count as the GPU path; rank 0 prints the line."""
+    import torch.distributed as dist
+
+    from paper_2608_11231_b200 import sharding
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    reqs = build_requests(args.workload, rank)
+    tokens = sum(r["total"] for r in reqs)
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(1e-3 * (rank + 1))
+    local_ms = 1e3 * (time.perf_counter() - t0) / args.steps
+    d = dist if world > 1 else None
+    ms = sharding.job_step_ms(local_ms, d)
+    total = sharding.job_total(tokens, d)
+    if rank == 0:
+        print(json.dumps(dict(metric=METRIC, value=total / (ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
+                              warmup=args.warmup, ms_per_step=ms, higher_is_better=True, scaling="weak",
+                              vs_baseline=None, dtype="none", data="none (stand-in step on CPU)",
+                              config=dict(workload=args.workload, requests=len(reqs), context_tokens=total,
+                                          dry_run=True), gpu_launches=0)))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -635,7 +785,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="composition time against K instead of the step benchmark")
     ap.add_argument("--artifacts", action="store_true", help="time of building chunk states and transitions")
+    ap.add_argument("--no-configs", action="store_true", help="leave the cfg1-cfg3 object out of the default line")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="ranks on CPU over gloo with a stand-in step: exercises the launch, sharding and timing "
+                         "reduction of --gpus N where there are no GPUs")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain script: become the launcher of N ranks of this same command line, one per GPU
+        from paper_2608_11231_b200 import sharding
+        sys.exit(sharding.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
+    if args.dry_run:
+        run_dry(args)
+        return
     if args.artifacts:
         run_artifacts(args)
     elif args.sweep:

@@ -41,3 +41,21 @@ def job_total(local_count: int, dist=None, device=None) -> int:
     t = torch.tensor([int(local_count)], dtype=torch.int64, device=device if device is not None else "cpu")
     dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return int(t.item())
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def launch_ranks(script: str, argv, n: int, timeout=None) -> int:
+    """Runs `script argv` as n ranks on this node (torch.distributed.run, rendezvous on 127.0.0.1, a free port):
+    RANK / LOCAL_RANK / WORLD_SIZE reach every rank through the environment.  Returns the launcher's exit code;
+    the ranks' output goes to this process's stdout / stderr."""
+    import subprocess
+    import sys
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={int(n)}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script] + list(argv)
+    return subprocess.run(cmd, timeout=timeout).returncode

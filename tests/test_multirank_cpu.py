@@ -50,3 +50,23 @@ def test_two_ranks_shard_requests_and_reduce_time():
 def test_single_rank_needs_no_process_group():
     assert sharding.job_step_ms(3.5) == 3.5 and sharding.job_total(7) == 7
     assert len(sharding.rank_requests("cfg3", 0)) == 8
+
+
+def test_bench_launches_its_own_ranks():
+    """`bench.py --gpus 2` started as a plain script becomes the launcher of two ranks; with --dry-run the ranks are
+    gloo processes on CPU with a stand-in step (rank r sleeps r + 1 ms), everything else is the benchmark's own path."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "5", "--warmup", "1",
+                        "--dry-run"], capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                               # rank 0 alone prints
+    line = json.loads(lines[0])
+    tokens = sum(q["total"] for rank in range(2) for q in sharding.rank_requests("cfg4", rank))
+    assert line["n_gpus"] == 2 and line["config"]["context_tokens"] == tokens
+    assert line["ms_per_step"] >= 2.0                    # the slow rank's time, not rank 0's
+    assert abs(line["value"] - tokens / (line["ms_per_step"] * 1e-3)) <= 1e-6 * line["value"]
