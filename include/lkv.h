@@ -25,8 +25,8 @@
  *     launched and copied to the device by the call itself (into the
  *     caller's workspace).  They may be reused as soon as the call returns.
  *     A list that fits the kernel parameters (n_req + 1 + selection indices +
- *     chunk ids <= 4000 ints for the initialisers, n_seq + 1 <= 1000 for the
- *     scans) travels inside the launch and the call may be captured into a
+ *     chunk ids <= 4000 ints for the initialisers, 2 n_seq + 1 <= 1000 for the
+ *     scans, which send the launch order along: longest sequence first) travels inside the launch and the call may be captured into a
  *     CUDA graph; a longer list needs a host-to-device copy of an array that
  *     dies with the call, so such a call returns LKV_ERR_UNSUPPORTED while
  *     `stream` is capturing.

@@ -139,6 +139,7 @@ def _hp(a: Optional[np.ndarray]):
 
 
 _ws_cache = {}
+_err_ws_cache = {}
 
 
 def workspace(device, nbytes: int) -> torch.Tensor:
@@ -340,7 +341,11 @@ def lkv_state_rel_error(S_init, S_ref, n_states: Optional[int] = None, rel_err=N
     if rel_err is None:
         rel_err = torch.empty((n,), dtype=torch.float32, device=S_init.device)
     nbytes = load().lkv_state_rel_error_workspace_bytes(n, elems)
-    ws_t = workspace(S_init.device, max(int(nbytes), 256))
+    # scratch of its own: this call keeps partial sums from byte 0 on, it has no status header
+    key = torch.device(S_init.device).index
+    ws_t = _err_ws_cache.get(key)
+    if ws_t is None or ws_t.numel() < nbytes:
+        ws_t = _err_ws_cache[key] = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=S_init.device)
     st = load().lkv_state_rel_error(_ptr(S_init), _ptr(S_ref), _ptr(rel_err), n, elems, ws_t.data_ptr(), ws_t.numel(),
                                     _stream(stream))
     if st != LKV_OK:

@@ -40,7 +40,7 @@ struct IndexBlock {
     __device__ __forceinline__ int32_t operator[](int i) const { return ptr ? ptr[i] : v[i]; }
 };
 constexpr int kInitIdxCap = 4000;  // ints: cu_k | sel | ids
-constexpr int kScanIdxCap = 1000;  // ints: cu_seqlens
+constexpr int kScanIdxCap = 1000;  // ints: cu_seqlens[n_seq + 1] | launch order[n_seq]
 
 // Launch-side records shared by the entry points and the kernels.  Passed by value as
 // __grid_constant__ kernel parameters.
@@ -68,7 +68,7 @@ struct GdnArgs {
     int32_t s0_identity;         // start every sequence from S = I (d_k == d_v) instead of S0; with v == nullptr (read
                                  // as zeros) the final state is then the sequence's accumulated transition; o may be nullptr
     int32_t *status;
-    IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]
+    IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1], then the launch order: sequence of grid row y at [n_seq + 1 + y]
 };
 
 struct SsdArgs {

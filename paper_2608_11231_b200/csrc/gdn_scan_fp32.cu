@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
     float *bs = cg + kC;                   // [kC]
     float *gs = bs + kC;                   // [kC]
 
-    const int h = blockIdx.x, seq = blockIdx.y;
+    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
     const int hk = h / (a.H_v / a.H_k);
     const int tid = threadIdx.x;
     const int j = tid % DV, tg = tid / DV;

@@ -271,7 +271,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     __shared__ volatile int dead;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.x, seq = blockIdx.y;
+    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
     const int hk = h / (a.H_v / a.H_k);
     const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
     const int nblk = (t_end - t_begin + kC - 1) / kC;

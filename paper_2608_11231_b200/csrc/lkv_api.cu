@@ -2,6 +2,7 @@
 // Everything that can be wrong with a call is found here, on the host, before a launch.
 #include <string.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -170,6 +171,16 @@ int check_seqs(int T_total, int n_seq, const int32_t *cu_seqlens, std::vector<in
     return LKV_OK;
 }
 
+// Appends to cu[n_seq + 1] the launch order of the sequences: longest first (ties by index), so that the CTAs of the
+// long sequences, which are scheduled in grid order, start first and the short ones fill the tail of the launch.
+void append_launch_order(std::vector<int32_t> &cu, int n_seq) {
+    std::vector<int32_t> order(n_seq);
+    for (int i = 0; i < n_seq; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(),
+                     [&](int32_t x, int32_t y) { return cu[x + 1] - cu[x] > cu[y + 1] - cu[y]; });
+    cu.insert(cu.end(), order.begin(), order.end());
+}
+
 }  // namespace
 
 extern "C" {
@@ -213,7 +224,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(S0) ||
         !aligned16(o) || !aligned16(S_T))
         return LKV_ERR_ALIGN;
-    if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(2 * d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
     if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
     {
         // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
@@ -250,6 +261,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         use_tensor = tensor_fits;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    append_launch_order(cu, d->n_seq);
     st = place_indices(a.cu, cu, d->workspace, s);
     if (st != LKV_OK) return st;
     const cudaError_t e = use_tensor ? launch_gdn_scan_tensor(a, s) : launch_gdn_scan_fp32(a, io_bf16, s);
@@ -320,7 +332,7 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
     if (!aligned16(x) || !aligned16(dt) || !aligned16(A) || !aligned16(B) || !aligned16(C) || !aligned16(S0) ||
         !aligned16(y) || !aligned16(S_T))
         return LKV_ERR_ALIGN;
-    if (!d->workspace || d->workspace_bytes < ws_bytes_for(d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
+    if (!d->workspace || d->workspace_bytes < ws_bytes_for(2 * d->n_seq + 1, kScanIdxCap)) return LKV_ERR_WORKSPACE;
     if (!aligned16(d->workspace)) return LKV_ERR_ALIGN;
     {
         // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
@@ -355,6 +367,7 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
         use_tensor = tensor_fits;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    append_launch_order(cu, d->n_seq);
     st = place_indices(a.cu, cu, d->workspace, s);
     if (st != LKV_OK) return st;
     const cudaError_t e = use_tensor ? launch_ssd_scan_tensor(a, s) : launch_ssd_scan_fp32(a, io_bf16, s);
@@ -366,7 +379,7 @@ size_t lkv_workspace_bytes(int which, const void *desc, int n_units, int n_index
     switch (which) {
         case LKV_WS_INIT: return ws_bytes_for(2 * n_units + 1 + n_index, kInitIdxCap);
         case LKV_WS_GDN:
-        case LKV_WS_SSD: return ws_bytes_for(n_units + 1, kScanIdxCap);
+        case LKV_WS_SSD: return ws_bytes_for(2 * n_units + 1, kScanIdxCap);
         default: return 0;
     }
 }

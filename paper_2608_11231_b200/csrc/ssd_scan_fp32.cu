@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(256) ssd_scan_fp32_kernel(const __grid_constan
     float *ls = Gm + kQ * (kQ + 1);   // [kQ]
     float *dts = ls + kQ;             // [kQ]
 
-    const int h = blockIdx.x, seq = blockIdx.y;
+    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
     const int grp = h / (a.H / a.G);
     const int tid = threadIdx.x;
     const int p = tid % P, tg = tid / P;

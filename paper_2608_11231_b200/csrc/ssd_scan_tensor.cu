@@ -85,7 +85,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
     __shared__ float scan_carry[4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.x, seq = blockIdx.y;
+    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
     const int grp = h / (a.H / a.G);
     const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
     const int nblk = (t_end - t_begin + kQ - 1) / kQ;
