@@ -136,7 +136,8 @@ typedef struct lkv_init_desc {
  *   q, k   [T_total, H_k, d_k]   io_dtype        v  [T_total, H_v, d_v]  io_dtype
  *   g      float [T_total, H_v]  log-decay, alpha = exp(g) <= 1 expected
  *   beta   float [T_total, H_v]
- *   S0,S_T float [n_seq, H_v, d_k, d_v]          o  [T_total, H_v, d_v]  io_dtype
+ *   S0     float [n_seq, H_v, d_k, d_v]          o  [T_total, H_v, d_v]  io_dtype
+ *   S_T    [n_seq, H_v, d_k, d_v] state_dtype (fp32, or bf16 as a cache pool stores states)
  * Value head h reads q/k head h / (H_v / H_k).
  */
 typedef struct lkv_gdn_desc {
@@ -150,7 +151,7 @@ typedef struct lkv_gdn_desc {
     int32_t io_dtype;          /* dtype of q, k, v and o */
     int32_t compute;           /* LKV_COMPUTE_* */
     float scale;               /* read-out scale; 0 selects d_k^(-1/2) */
-    int32_t reserved;
+    int32_t state_dtype;       /* dtype of S_T: LKV_DTYPE_F32 (0) or LKV_DTYPE_BF16; S0 is always fp32 */
     void *workspace;
     size_t workspace_bytes;
 } lkv_gdn_desc;
@@ -159,7 +160,8 @@ typedef struct lkv_gdn_desc {
  * Descriptor of lkv_ssd_fwd.
  *   x  [T_total, H, P] io_dtype      dt float [T_total, H] (already activated, > 0)
  *   A  float [H] (< 0)               B, C [T_total, G, N] io_dtype
- *   S0,S_T float [n_seq, H, N, P]    y  [T_total, H, P] io_dtype
+ *   S0 float [n_seq, H, N, P]        y  [T_total, H, P] io_dtype
+ *   S_T [n_seq, H, N, P] state_dtype (fp32, or bf16 as a cache pool stores states)
  * Head h reads group h / (H / G).
  */
 typedef struct lkv_ssd_desc {
@@ -172,6 +174,7 @@ typedef struct lkv_ssd_desc {
     int32_t G;                 /* groups, divides H */
     int32_t io_dtype;
     int32_t compute;
+    int32_t state_dtype;       /* dtype of S_T: LKV_DTYPE_F32 (0) or LKV_DTYPE_BF16; S0 is always fp32 */
     void *workspace;
     size_t workspace_bytes;
 } lkv_ssd_desc;
@@ -270,7 +273,7 @@ int lkv_device_status_static(void *stream);
  * any length >= 0 are accepted (no padding is required).
  */
 int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
-                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream);
+                const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream);
 
 /*
  * Mamba-2 (SSD) scan from an initial state (Eq. 1 with Eq. 2; Algorithm 1, line 3).
@@ -280,7 +283,7 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
  * NULL conventions as in lkv_gdn_fwd.
  */
 int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
-                const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream);
+                const float *S0, void *y, void *S_T, const lkv_ssd_desc *d, void *stream);
 
 /*
  * Producers of the cached artefacts that exact composition consumes (Eq. 5: a chunk C maps an incoming
@@ -304,6 +307,24 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
 int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, float *transitions,
                              const lkv_gdn_desc *d, void *stream);
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream);
+
+/*
+ * GDN exact composition for ONE request WITHOUT materialised transitions (the "online fold": Eq. 6 evaluated as the
+ * chain of Eq. 5 with every T_C applied token by token from the chunk's cached key / gate stream):
+ *     S <- S_{c_1};   S <- (scan of chunk c_j's tokens with v = 0 from S) + S_{c_j},   j = 2..K.
+ * It trades the d_k x d_k fp32 transition per (chunk, head) for the chunk's k / g / beta stream and one scan per chunk.
+ *
+ *   states     fp32 pool [n_chunks, H, d_k, d_v] (d->state_dtype must be LKV_DTYPE_F32)
+ *   k          [total_tokens, H_k, d_k] io_dtype, the cached chunks' keys back to back in pool order
+ *   g, beta    float [total_tokens, H] as for lkv_gdn_fwd (H = d->H value heads)
+ *   cu_tokens  HOST int32[n_chunks + 1]: chunk c owns tokens cu_tokens[c] .. cu_tokens[c + 1]
+ *   K, d->chunk_ids, S0, d->workspace, d->compute as for lkv_init_state; d->family must be LKV_FAMILY_GDN, d_k == d_v.
+ * Launches 1 + (K - 1) kernels on `stream`.  The result equals lkv_init_state(..., LKV_INIT_EXACT) on transitions
+ * built by lkv_gdn_chunk_transition from the same streams, up to rounding.  Errors as for lkv_init_state and the scans.
+ */
+int lkv_init_state_fold(const void *states, const void *k, const float *g, const float *beta,
+                        const int32_t *cu_tokens, int K, void *S0, const lkv_init_desc *d, int H_k, int io_dtype,
+                        void *stream);
 
 /*
  * Diagnostic of Section 3.2 ("Diagnosis via relative error"): how far a constructed initial state is from the

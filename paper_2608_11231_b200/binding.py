@@ -28,7 +28,7 @@ LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
 LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
-           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_state_rel_error",
+           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_init_state_fold", "lkv_state_rel_error",
            "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_device_status_static",
            "lkv_selftest_bounded_wait", "lkv_status_string", "lkv_version")
 
@@ -44,14 +44,14 @@ class lkv_gdn_desc(ctypes.Structure):
     _fields_ = [("T_total", ctypes.c_int32), ("n_seq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p),
                 ("H_k", ctypes.c_int32), ("H_v", ctypes.c_int32), ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32),
                 ("io_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("scale", ctypes.c_float),
-                ("reserved", ctypes.c_int32), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("state_dtype", ctypes.c_int32), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
 class lkv_ssd_desc(ctypes.Structure):
     _fields_ = [("T_total", ctypes.c_int32), ("n_seq", ctypes.c_int32), ("cu_seqlens", ctypes.c_void_p),
                 ("H", ctypes.c_int32), ("P", ctypes.c_int32), ("N", ctypes.c_int32), ("G", ctypes.c_int32),
-                ("io_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("workspace", ctypes.c_void_p),
-                ("workspace_bytes", ctypes.c_size_t)]
+                ("io_dtype", ctypes.c_int32), ("compute", ctypes.c_int32), ("state_dtype", ctypes.c_int32),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
 class LkvError(RuntimeError):
@@ -80,6 +80,8 @@ def load() -> ctypes.CDLL:
         lib.lkv_ssd_fwd.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_gdn_chunk_transition.argtypes = [vp] * 4 + [ctypes.POINTER(lkv_gdn_desc), vp]
         lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
+        lib.lkv_init_state_fold.argtypes = [vp, vp, vp, vp, vp, ci, vp, ctypes.POINTER(lkv_init_desc), ci, ci, vp]
+        lib.lkv_init_state_fold.restype = ci
         lib.lkv_state_rel_error.argtypes = [vp, vp, vp, ci, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
         lib.lkv_state_rel_error_workspace_bytes.argtypes = [ci, ctypes.c_size_t]
         lib.lkv_state_rel_error_workspace_bytes.restype = ctypes.c_size_t
@@ -240,24 +242,27 @@ def lkv_init_state_batched_static(states: torch.Tensor, transitions: Optional[to
 
 def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None, scale: float = 0.0,
                 compute: int = LKV_COMPUTE_AUTO, want_final_state: bool = True, want_outputs: bool = True,
-                workspace_t: Optional[torch.Tensor] = None, stream=None):
+                state_dtype=torch.float32, workspace_t: Optional[torch.Tensor] = None, stream=None):
     """Gated DeltaNet scan.  q, k: [T, H_k, d_k]; v: [T, H_v, d_v]; g, beta: [T, H_v] fp32.
 
-    Returns (o [T, H_v, d_v] in the dtype of v, or None with want_outputs=False; S_T [n_seq, H_v, d_k, d_v] fp32 or None).
+    Returns (o [T, H_v, d_v] in the dtype of v, or None with want_outputs=False; S_T [n_seq, H_v, d_k, d_v] in
+    state_dtype (fp32 or bf16; the dtype of S_T if one is passed) or None).
     """
     T, H_k, d_k = q.shape
     _, H_v, d_v = v.shape
     cu = _host_i32(cu_seqlens)
     n_seq = 1 if cu is None else cu.size - 1
     d = lkv_gdn_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H_k=H_k, H_v=H_v,
-                     d_k=d_k, d_v=d_v, io_dtype=_dtype_code(v), compute=compute, scale=float(scale), reserved=0,
+                     d_k=d_k, d_v=d_v, io_dtype=_dtype_code(v), compute=compute, scale=float(scale), state_dtype=0,
                      workspace=None, workspace_bytes=0)
     ws_t = workspace_t if workspace_t is not None else workspace(v.device, lkv_workspace_bytes(LKV_WS_GDN, d, n_seq))
     d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
     if o is None and want_outputs:
         o = torch.empty_like(v)
     if S_T is None and want_final_state:
-        S_T = torch.empty((n_seq, H_v, d_k, d_v), dtype=torch.float32, device=v.device)
+        S_T = torch.empty((n_seq, H_v, d_k, d_v), dtype=state_dtype, device=v.device)
+    if S_T is not None:
+        d.state_dtype = _dtype_code(S_T)
     st = load().lkv_gdn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S0), _ptr(o), _ptr(S_T),
                             ctypes.byref(d), _stream(stream))
     if st != LKV_OK:
@@ -266,11 +271,11 @@ def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None,
 
 
 def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, compute: int = LKV_COMPUTE_AUTO,
-                want_final_state: bool = True, want_outputs: bool = True,
+                want_final_state: bool = True, want_outputs: bool = True, state_dtype=torch.float32,
                 workspace_t: Optional[torch.Tensor] = None, stream=None):
     """Mamba-2 (SSD) scan.  x: [T, H, P]; dt: [T, H] fp32; A: [H] fp32; B, C: [T, G, N].
 
-    Returns (y [T, H, P] in the dtype of x, S_T [n_seq, H, N, P] fp32 or None).
+    Returns (y [T, H, P] in the dtype of x, S_T [n_seq, H, N, P] in state_dtype (fp32 or bf16) or None).
     """
     T, H, P = x.shape
     _, G, N = B.shape
@@ -283,12 +288,33 @@ def lkv_ssd_fwd(x, dt, A, B, C, S0=None, y=None, S_T=None, *, cu_seqlens=None, c
     if y is None and want_outputs:
         y = torch.empty_like(x)
     if S_T is None and want_final_state:
-        S_T = torch.empty((n_seq, H, N, P), dtype=torch.float32, device=x.device)
+        S_T = torch.empty((n_seq, H, N, P), dtype=state_dtype, device=x.device)
+    if S_T is not None:
+        d.state_dtype = _dtype_code(S_T)
     st = load().lkv_ssd_fwd(_ptr(x), _ptr(dt), _ptr(A), _ptr(B), _ptr(C), _ptr(S0), _ptr(y), _ptr(S_T),
                             ctypes.byref(d), _stream(stream))
     if st != LKV_OK:
         raise LkvError(st, "lkv_ssd_fwd")
     return y, S_T
+
+
+def lkv_init_state_fold(states: torch.Tensor, k, g, beta, cu_tokens, K: int, chunk_ids=None,
+                        S0: Optional[torch.Tensor] = None, *, compute: int = LKV_COMPUTE_AUTO,
+                        workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """GDN exact composition of one request from the cached key / gate streams (no materialised transitions).
+
+    states: fp32 pool [n_chunks, H, d, d]; k: [total_tokens, H_k, d]; g, beta: [total_tokens, H] fp32;
+    cu_tokens: host int32[n_chunks + 1].  Returns S0 [H, d, d] fp32.
+    """
+    ids, cu = _host_i32(chunk_ids), _host_i32(cu_tokens)
+    d, ws_t = _init_desc(states, LKV_FAMILY_GDN, compute, workspace_t, 1, int(K), ids)
+    if S0 is None:
+        S0 = torch.empty(tuple(states.shape[1:]), dtype=torch.float32, device=states.device)
+    st = load().lkv_init_state_fold(_ptr(states), _ptr(k), _ptr(g), _ptr(beta), _hp(cu), int(K), _ptr(S0),
+                                    ctypes.byref(d), int(k.shape[1]), _dtype_code(k), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_init_state_fold")
+    return S0
 
 
 def lkv_gdn_chunk_transition(k, g, beta, transitions=None, *, cu_seqlens=None, H_v: Optional[int] = None,
@@ -302,7 +328,7 @@ def lkv_gdn_chunk_transition(k, g, beta, transitions=None, *, cu_seqlens=None, H
     cu = _host_i32(cu_seqlens)
     n_seq = 1 if cu is None else cu.size - 1
     d = lkv_gdn_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H_k=H_k, H_v=H_v,
-                     d_k=d_k, d_v=d_k, io_dtype=_dtype_code(k), compute=compute, scale=0.0, reserved=0,
+                     d_k=d_k, d_v=d_k, io_dtype=_dtype_code(k), compute=compute, scale=0.0, state_dtype=0,
                      workspace=None, workspace_bytes=0)
     ws_t = workspace_t if workspace_t is not None else workspace(k.device, lkv_workspace_bytes(LKV_WS_GDN, d, n_seq))
     d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()

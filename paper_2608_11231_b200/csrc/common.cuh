@@ -30,6 +30,12 @@ __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <>
 __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
+// Final-state store of the scans: element idx of S_T as fp32, or rounded to bf16 when the caller asked for that.
+__device__ __forceinline__ void store_state(float *S_T, int st_bf16, size_t idx, float v) {
+    if (st_bf16) reinterpret_cast<__nv_bfloat16 *>(S_T)[idx] = __float2bfloat16_rn(v);
+    else S_T[idx] = v;
+}
+
 // Small host-checked index arrays travel to the device inside the kernel parameters
 // (no copy, no extra stream operation); lists longer than CAP are copied into the
 // caller's workspace instead and reached through `ptr`.
@@ -62,7 +68,9 @@ struct GdnArgs {
     const void *q, *k, *v;
     const float *g, *beta, *S0;
     void *o;
-    float *S_T;
+    float *S_T;                  // final states, fp32 or (st_bf16) bf16 behind the same pointer
+    const float *S_add;          // added to every final state before it is stored (Eq. 5: S_out = T_C S_in + S_local), or nullptr
+    int32_t st_bf16;
     int32_t n_seq, T_total, H_k, H_v, d_k, d_v;
     float scale;
     int32_t s0_identity;         // start every sequence from S = I (d_k == d_v) instead of S0; with v == nullptr (read
@@ -75,7 +83,8 @@ struct SsdArgs {
     const void *x, *B, *C;
     const float *dt, *A, *S0;
     void *y;
-    float *S_T;
+    float *S_T;                  // final states, fp32 or (st_bf16) bf16 behind the same pointer
+    int32_t st_bf16;
     int32_t n_seq, T_total, H, P, N, G;
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1]

@@ -279,9 +279,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     const bool has_v = a.v != nullptr, has_o = a.o != nullptr;
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
-        if (a.S_T && (a.S_T != a.S0 || a.s0_identity))
+        if (a.S_T && (a.S_T != a.S0 || a.s0_identity || a.S_add))
             for (int e = tid; e < kD * kD; e += kThreads)
-                a.S_T[sbase + e] = a.s0_identity ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f);
+                store_state(a.S_T, a.st_bf16, sbase + e,
+                            (a.s0_identity ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f)) +
+                                (a.S_add ? a.S_add[sbase + e] : 0.f));
         return;
     }
     if (tid == 0) {
@@ -853,8 +855,10 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                         tmem_ld16(lane_base + kTmS + 64 * half + 16 * q, rr);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int c = 0; c < 16; ++c)
-                            a.S_T[sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j] = __uint_as_float(rr[c]);
+                        for (int c = 0; c < 16; ++c) {
+                            const size_t e = sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j;
+                            store_state(a.S_T, a.st_bf16, e, __uint_as_float(rr[c]) + (a.S_add ? a.S_add[e] : 0.f));
+                        }
                     }
                 }
             } else {

@@ -208,10 +208,16 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
 }
 
 // lkv_gdn_fwd, and with `transition` set the scan from S = I with v = 0 whose final state is the chunk transition
+// what: 0 = scan, 1 = chunk transitions (start from S = I, v read as zeros), 2 = one step of the online fold (v read as
+// zeros, S_add added to the final state)
 static int gdn_impl(const void *q, const void *k, const void *v, const float *g, const float *beta,
-                    const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream, bool transition) {
+                    const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream, int what,
+                    const float *S_add = nullptr) {
+    const bool transition = what == 1;
     if (!d) return LKV_ERR_NULL;
-    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
+    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute) || !dtype_ok(d->state_dtype)) return LKV_ERR_MODE;
+    const bool st_bf16 = d->state_dtype == LKV_DTYPE_BF16;
+    if (st_bf16 && S_T && S_T == S0) return LKV_ERR_OVERLAP;   // an fp32 input cannot be a bf16 output
     if (d->H_k < 1 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1 || d->H_v % d->H_k != 0) return LKV_ERR_DIM;
     std::vector<int32_t> cu;
     int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
@@ -219,7 +225,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     if (d->n_seq == 0) return LKV_OK;
     if (transition && d->d_k != d->d_v) return LKV_ERR_DIM;
     if (d->T_total > 0 && (!q || !k || !g || !beta)) return LKV_ERR_NULL;
-    if (!transition && d->T_total > 0 && !v) return LKV_ERR_NULL;
+    if (what == 0 && d->T_total > 0 && !v) return LKV_ERR_NULL;
     if (!o && !S_T) return LKV_ERR_NULL;   // nothing to compute
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(g) || !aligned16(beta) || !aligned16(S0) ||
         !aligned16(o) || !aligned16(S_T))
@@ -230,9 +236,10 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
         const size_t es = d->io_dtype == LKV_DTYPE_BF16 ? 2 : 4, T = static_cast<size_t>(d->T_total);
         const size_t qk_b = es * T * d->H_k * d->d_k, v_b = es * T * d->H_v * d->d_v, gb_b = sizeof(float) * T * d->H_v;
-        const size_t st_b = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H_v * d->d_k * d->d_v;
+        const size_t st_in = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H_v * d->d_k * d->d_v;
+        const size_t st_b = st_bf16 ? st_in / 2 : st_in;
         const void *in[6] = {q, k, v, g, beta, S0};
-        const size_t in_b[6] = {qk_b, qk_b, v ? v_b : 0, gb_b, gb_b, S0 ? st_b : 0};
+        const size_t in_b[6] = {qk_b, qk_b, v ? v_b : 0, gb_b, gb_b, S0 ? st_in : 0};
         for (int i = 0; i < 6; ++i) {
             if (overlaps(o, o ? v_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
             if (!(i == 5 && S_T == S0) && overlaps(S_T, S_T ? st_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
@@ -241,7 +248,8 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     }
 
     GdnArgs a;
-    a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = S_T;
+    a.q = q; a.k = k; a.v = v; a.g = g; a.beta = beta; a.S0 = S0; a.o = o; a.S_T = static_cast<float *>(S_T);
+    a.S_add = S_add; a.st_bf16 = st_bf16 ? 1 : 0;
     a.n_seq = d->n_seq; a.T_total = d->T_total; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
     a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
     a.s0_identity = transition ? 1 : 0;
@@ -269,15 +277,58 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
 }
 
 int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, const float *beta,
-                const float *S0, void *o, float *S_T, const lkv_gdn_desc *d, void *stream) {
-    return gdn_impl(q, k, v, g, beta, S0, o, S_T, d, stream, false);
+                const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream) {
+    return gdn_impl(q, k, v, g, beta, S0, o, S_T, d, stream, 0);
 }
 
 int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, float *transitions,
                              const lkv_gdn_desc *d, void *stream) {
     if (d && d->n_seq > 0 && !transitions) return LKV_ERR_NULL;
     // q is not needed for the state: the key tensor stands in for it (its read-outs are not written)
-    return gdn_impl(k, k, nullptr, g, beta, nullptr, nullptr, transitions, d, stream, true);
+    if (d && d->state_dtype != LKV_DTYPE_F32) return LKV_ERR_MODE;   // transitions are fp32
+    return gdn_impl(k, k, nullptr, g, beta, nullptr, nullptr, transitions, d, stream, 1);
+}
+
+int lkv_init_state_fold(const void *states, const void *k, const float *g, const float *beta,
+                        const int32_t *cu_tokens, int K, void *S0, const lkv_init_desc *d, int H_k, int io_dtype,
+                        void *stream) {
+    int st = check_init_desc(d);
+    if (st != LKV_OK) return st;
+    if (d->family != LKV_FAMILY_GDN || !dtype_ok(io_dtype)) return LKV_ERR_MODE;
+    if (d->state_dtype != LKV_DTYPE_F32) return LKV_ERR_UNSUPPORTED;   // the cached states are added in fp32
+    if (K < 0 || H_k < 1 || d->H % H_k != 0 || d->d_k != d->d_v) return LKV_ERR_DIM;
+    if (!states || !S0 || !cu_tokens) return LKV_ERR_NULL;
+    if (K > 0 && !d->chunk_ids && K > d->n_chunks) return LKV_ERR_INDEX;
+    if (cu_tokens[0] != 0) return LKV_ERR_INDEX;
+    for (int c = 0; c < d->n_chunks; ++c)
+        if (cu_tokens[c + 1] < cu_tokens[c]) return LKV_ERR_INDEX;
+    std::vector<int32_t> ids(K);
+    for (int j = 0; j < K; ++j) {
+        ids[j] = d->chunk_ids ? d->chunk_ids[j] : j;
+        if (ids[j] < 0 || ids[j] >= d->n_chunks) return LKV_ERR_INDEX;
+    }
+    if (K >= 2 && cu_tokens[d->n_chunks] > 0 && (!k || !g || !beta)) return LKV_ERR_NULL;
+    // the first chunk's state (or the zero state) through the single-state path, then one scan per later chunk
+    lkv_init_desc first = *d;
+    first.sel_index = 0;
+    st = lkv_init_state(states, nullptr, K, LKV_INIT_INDEX, S0, &first, stream);
+    if (st != LKV_OK) return st;
+    const size_t es = io_dtype == LKV_DTYPE_BF16 ? 2 : 4;
+    const size_t state_elems = static_cast<size_t>(d->H) * d->d_k * d->d_v;
+    for (int j = 1; j < K; ++j) {
+        const int c = ids[j], t0 = cu_tokens[c], len = cu_tokens[c + 1] - t0;
+        lkv_gdn_desc sd{};
+        sd.T_total = len; sd.n_seq = 1; sd.cu_seqlens = nullptr; sd.H_k = H_k; sd.H_v = d->H; sd.d_k = d->d_k; sd.d_v = d->d_v;
+        sd.io_dtype = io_dtype; sd.compute = d->compute; sd.scale = 0.f; sd.state_dtype = LKV_DTYPE_F32;
+        sd.workspace = d->workspace; sd.workspace_bytes = d->workspace_bytes;
+        const char *kc = static_cast<const char *>(k) + es * static_cast<size_t>(t0) * H_k * d->d_k;
+        const float *gc = g ? g + static_cast<size_t>(t0) * d->H : nullptr;
+        const float *bc = beta ? beta + static_cast<size_t>(t0) * d->H : nullptr;
+        st = gdn_impl(kc, kc, nullptr, gc, bc, static_cast<const float *>(S0), nullptr, S0, &sd, stream, 2,
+                      static_cast<const float *>(states) + static_cast<size_t>(c) * state_elems);
+        if (st != LKV_OK) return st;
+    }
+    return LKV_OK;
 }
 
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream) {
@@ -318,9 +369,11 @@ int lkv_state_rel_error(const float *S_init, const float *S_ref, float *rel_err,
 }
 
 int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, const void *C,
-                const float *S0, void *y, float *S_T, const lkv_ssd_desc *d, void *stream) {
+                const float *S0, void *y, void *S_T, const lkv_ssd_desc *d, void *stream) {
     if (!d) return LKV_ERR_NULL;
-    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute)) return LKV_ERR_MODE;
+    if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute) || !dtype_ok(d->state_dtype)) return LKV_ERR_MODE;
+    const bool st_bf16 = d->state_dtype == LKV_DTYPE_BF16;
+    if (st_bf16 && S_T && S_T == S0) return LKV_ERR_OVERLAP;   // an fp32 input cannot be a bf16 output
     if (d->H < 1 || d->P < 1 || d->N < 1 || d->G < 1 || d->H % d->G != 0) return LKV_ERR_DIM;
     std::vector<int32_t> cu;
     int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
@@ -338,9 +391,10 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
         // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
         const size_t es = d->io_dtype == LKV_DTYPE_BF16 ? 2 : 4, T = static_cast<size_t>(d->T_total);
         const size_t x_b = es * T * d->H * d->P, bc_b = es * T * d->G * d->N, dt_b = sizeof(float) * T * d->H;
-        const size_t st_b = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H * d->N * d->P;
+        const size_t st_in = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H * d->N * d->P;
+        const size_t st_b = st_bf16 ? st_in / 2 : st_in;
         const void *in[6] = {x, dt, A, B, C, S0};
-        const size_t in_b[6] = {x_b, dt_b, sizeof(float) * d->H, bc_b, bc_b, S0 ? st_b : 0};
+        const size_t in_b[6] = {x_b, dt_b, sizeof(float) * d->H, bc_b, bc_b, S0 ? st_in : 0};
         for (int i = 0; i < 6; ++i) {
             if (overlaps(y, y ? x_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
             if (!(i == 5 && S_T == S0) && overlaps(S_T, S_T ? st_b : 0, in[i], in_b[i])) return LKV_ERR_OVERLAP;
@@ -349,7 +403,8 @@ int lkv_ssd_fwd(const void *x, const float *dt, const float *A, const void *B, c
     }
 
     SsdArgs a;
-    a.x = x; a.dt = dt; a.A = A; a.B = B; a.C = C; a.S0 = S0; a.y = y; a.S_T = S_T;
+    a.x = x; a.dt = dt; a.A = A; a.B = B; a.C = C; a.S0 = S0; a.y = y; a.S_T = static_cast<float *>(S_T);
+    a.st_bf16 = st_bf16 ? 1 : 0;
     a.n_seq = d->n_seq; a.T_total = d->T_total; a.H = d->H; a.P = d->P; a.N = d->N; a.G = d->G;
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;

@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(256) ssd_scan_fp32_kernel(const __grid_constan
     }
     if (a.S_T) {
         __syncthreads();
-        for (int idx = tid; idx < N * P; idx += 256) a.S_T[sbase + idx] = S[idx];
+        for (int idx = tid; idx < N * P; idx += 256) store_state(a.S_T, a.st_bf16, sbase + idx, S[idx]);
     }
 }
 

@@ -93,7 +93,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
         if (a.S_T && a.S_T != a.S0)
-            for (int e = tid; e < kN * kP; e += kThreads) a.S_T[sbase + e] = a.S0 ? a.S0[sbase + e] : 0.f;
+            for (int e = tid; e < kN * kP; e += kThreads) store_state(a.S_T, a.st_bf16, sbase + e, a.S0 ? a.S0[sbase + e] : 0.f);
         return;
     }
     if (tid == 0) {
@@ -330,7 +330,14 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
                 tmem_ld32(lane_base + kTmH + 32 * q, rr);
                 tmem_ld_wait();
                 if (last) {
-                    if (a.S_T && !dead) {
+                    if (a.S_T && !dead && a.st_bf16) {
+                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(a.S_T) + sbase + static_cast<size_t>(x) * kP + 32 * q;
+#pragma unroll
+                        for (int c = 0; c < 32; c += 8)
+                            *reinterpret_cast<uint4 *>(dst + c) =
+                                make_uint4(pack_bf16(__uint_as_float(rr[c]), __uint_as_float(rr[c + 1])), pack_bf16(__uint_as_float(rr[c + 2]), __uint_as_float(rr[c + 3])),
+                                           pack_bf16(__uint_as_float(rr[c + 4]), __uint_as_float(rr[c + 5])), pack_bf16(__uint_as_float(rr[c + 6]), __uint_as_float(rr[c + 7])));
+                    } else if (a.S_T && !dead) {
 #pragma unroll
                         for (int c = 0; c < 32; c += 4)
                             *reinterpret_cast<float4 *>(a.S_T + sbase + static_cast<size_t>(x) * kP + 32 * q + c) =

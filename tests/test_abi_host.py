@@ -102,7 +102,7 @@ def test_init_state_batched_argument_errors(lib):
 
 def _gdn_desc(**kw):
     base = dict(T_total=100, n_seq=1, cu_seqlens=None, H_k=2, H_v=4, d_k=64, d_v=64, io_dtype=b.LKV_DTYPE_F32,
-                compute=b.LKV_COMPUTE_AUTO, scale=0.0, reserved=0, workspace=FAKE, workspace_bytes=1 << 20)
+                compute=b.LKV_COMPUTE_AUTO, scale=0.0, state_dtype=0, workspace=FAKE, workspace_bytes=1 << 20)
     base.update(kw)
     return b.lkv_gdn_desc(**base)
 
@@ -127,6 +127,8 @@ def test_gdn_fwd_argument_errors(lib):
     assert f(_gdn_desc(), o=fake(1) + 1024) == b.LKV_ERR_OVERLAP           # o inside q
     assert f(_gdn_desc(), S0=fake(6), S_T=fake(6) + 256) == b.LKV_ERR_OVERLAP   # S_T may be S0 itself, not a shifted view
     assert f(_gdn_desc(), S_T=fake(4)) == b.LKV_ERR_OVERLAP                # S_T on g
+    assert f(_gdn_desc(state_dtype=7)) == b.LKV_ERR_MODE
+    assert f(_gdn_desc(state_dtype=b.LKV_DTYPE_BF16), S0=fake(6), S_T=fake(6)) == b.LKV_ERR_OVERLAP   # fp32 in, bf16 out
     assert f(_gdn_desc(d_v=48)) == b.LKV_ERR_UNSUPPORTED
     assert f(_gdn_desc(workspace=None)) == b.LKV_ERR_WORKSPACE
     assert f(_gdn_desc(compute=b.LKV_COMPUTE_TENSOR, d_k=24, d_v=32)) == b.LKV_ERR_UNSUPPORTED
@@ -219,3 +221,27 @@ def test_selftest_and_static_status_argument_errors(lib):
     assert lib.lkv_selftest_bounded_wait(0, FAKE, None) == b.LKV_ERR_DIM
     assert lib.lkv_selftest_bounded_wait(1 << 21, FAKE, None) == b.LKV_ERR_DIM
     assert lib.lkv_selftest_bounded_wait(1000, FAKE + 4, None) == b.LKV_ERR_ALIGN
+
+
+def test_fold_argument_errors(lib):
+    cu = np.array([0, 100, 300, 300], dtype=np.int32)
+    ids = np.array([2, 0, 1], dtype=np.int32)
+
+    def call(d, K=3, states=fake(1), k=fake(2), cu_p=cu.ctypes.data, S0=fake(5), H_k=2, io=b.LKV_DTYPE_BF16):
+        return lib.lkv_init_state_fold(states, k, fake(3), fake(4), cu_p, K, S0, ctypes.byref(d) if d is not None else None,
+                                       H_k, io, None)
+    gd = lambda **kw: _desc(**dict(dict(family=b.LKV_FAMILY_GDN, H=4, d_k=64, d_v=64, n_chunks=3, chunk_ids=ids.ctypes.data), **kw))
+    assert call(None) == b.LKV_ERR_NULL
+    assert call(_desc(family=b.LKV_FAMILY_MAMBA2, n_chunks=3)) == b.LKV_ERR_MODE      # Mamba-2 has no key stream to fold
+    assert call(gd(), io=9) == b.LKV_ERR_MODE
+    assert call(gd(state_dtype=b.LKV_DTYPE_BF16)) == b.LKV_ERR_UNSUPPORTED
+    assert call(gd(), K=-1) == b.LKV_ERR_DIM
+    assert call(gd(), H_k=3) == b.LKV_ERR_DIM
+    assert call(gd(d_v=32)) == b.LKV_ERR_DIM
+    assert call(gd(), states=None) == b.LKV_ERR_NULL
+    assert call(gd(), cu_p=None) == b.LKV_ERR_NULL
+    assert call(gd(), k=None) == b.LKV_ERR_NULL
+    bad = np.array([0, 100, 50, 300], dtype=np.int32)
+    assert call(gd(), cu_p=bad.ctypes.data) == b.LKV_ERR_INDEX
+    ids[1] = 3
+    assert call(gd()) == b.LKV_ERR_INDEX

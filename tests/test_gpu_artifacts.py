@@ -156,3 +156,60 @@ def test_state_rel_error_of_the_two_initialisers():
     e_lb = host(b.lkv_state_rel_error(S_lb, S_star, n_states=1))[0]
     assert e_ex <= 2e-2 and e_lb > 5 * e_ex
 
+
+
+def test_online_fold_equals_exact_composition_and_one_pass():
+    """Eq. 6 without materialised transitions: S <- scan_{v=0}(chunk j's keys and gates; from S) + S_j.
+    Equals the composition over materialised transitions and, by the paper's identity, the state of one pass over
+    the concatenated prefix."""
+    import torch
+    from helpers import TOL_BF16, dev, host, maxrel
+    rng = np.random.default_rng(41)
+    H_k, H_v, d = 2, 4, 128
+    lens = [200, 64, 0, 131, 77]                      # cached chunks in pool order (one of them empty)
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    tok = wl.gdn_tokens(rng, int(cu[-1]), H_k, H_v, d, d, io="bf16", live_chunk_len=128)
+    bf = torch.bfloat16
+    k, g, beta = dev(tok["k"], bf), dev(tok["g"]), dev(tok["beta"])
+    # the cache as the library builds it: local states (scan from the empty state) and transitions, fp32
+    _, states = b.lkv_gdn_fwd(dev(tok["q"], bf), k, dev(tok["v"], bf), g, beta, cu_seqlens=cu, want_outputs=False)
+    trans = b.lkv_gdn_chunk_transition(k, g, beta, cu_seqlens=cu)
+    ids = np.array([3, 0, 2, 4, 1], dtype=np.int32)   # a request that uses the chunks in another order
+    for compute in (b.LKV_COMPUTE_AUTO, b.LKV_COMPUTE_FP32):
+        S_fold = b.lkv_init_state_fold(states, k, g, beta, cu, len(ids), ids, compute=compute)
+        S_mat = b.lkv_init_state(states, trans, len(ids), b.LKV_INIT_EXACT, family=b.LKV_FAMILY_GDN, chunk_ids=ids)
+        assert maxrel(host(S_fold), host(S_mat)) <= TOL_BF16
+        # one pass of the oracle over the chunks' tokens in request order
+        order = np.concatenate([np.arange(cu[c], cu[c + 1]) for c in ids])
+        _, S_ref = oracle.gdn_seq(tok["q"][order], tok["k"][order], tok["v"][order], tok["g"][order], tok["beta"][order])
+        assert maxrel(host(S_fold), S_ref) <= TOL_BF16
+    # K = 1 is the stored state, K = 0 the zero state
+    assert torch.equal(b.lkv_init_state_fold(states, k, g, beta, cu, 1, ids[:1]), states[3])
+    assert float(b.lkv_init_state_fold(states, k, g, beta, cu, 0, None).abs().max()) == 0.0
+
+
+def test_final_states_stored_as_bf16_are_the_rounded_fp32_ones():
+    import torch
+    from helpers import dev, host
+    rng = np.random.default_rng(42)
+    bf = torch.bfloat16
+    lens = [150, 0, 64]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    tok = wl.gdn_tokens(rng, int(cu[-1]), 2, 4, 128, 128, io="bf16", live_chunk_len=64)
+    S0 = dev(rng.standard_normal((3, 4, 128, 128)).astype(np.float32))
+    a = (dev(tok["q"], bf), dev(tok["k"], bf), dev(tok["v"], bf), dev(tok["g"]), dev(tok["beta"]), S0)
+    for compute in (b.LKV_COMPUTE_TENSOR, b.LKV_COMPUTE_FP32):
+        _, S32 = b.lkv_gdn_fwd(*a, cu_seqlens=cu, compute=compute, want_outputs=False)
+        _, S16 = b.lkv_gdn_fwd(*a, cu_seqlens=cu, compute=compute, want_outputs=False, state_dtype=bf)
+        assert S16.dtype == bf and torch.equal(S16, S32.to(bf))
+    A = wl.ssd_A(rng, 3, live_chunk_len=64)
+    mt = wl.ssd_tokens(rng, int(cu[-1]), 3, 64, 128, 1)
+    M0 = dev(rng.standard_normal((3, 3, 128, 64)).astype(np.float32))
+    m = (dev(mt["x"], bf), dev(mt["dt"]), dev(A), dev(mt["B"], bf), dev(mt["C"], bf), M0)
+    for compute in (b.LKV_COMPUTE_TENSOR, b.LKV_COMPUTE_FP32):
+        _, S32 = b.lkv_ssd_fwd(*m, cu_seqlens=cu, compute=compute, want_outputs=False)
+        _, S16 = b.lkv_ssd_fwd(*m, cu_seqlens=cu, compute=compute, want_outputs=False, state_dtype=bf)
+        assert S16.dtype == bf and torch.equal(S16, S32.to(bf))
+    # a bf16 pool built this way feeds the initialisers
+    S_last = b.lkv_init_state(S16, None, 3, b.LKV_INIT_LAST, family=b.LKV_FAMILY_MAMBA2)
+    assert torch.equal(S_last, S16[2].float())
