@@ -63,7 +63,7 @@ def ssd_scan_flops(tokens: int, s=SSD_SHAPE, Q=SSD_BLOCK) -> float:
 # DRAM bytes (read + write) per scanned token from ncu captures of one launch of each scan kernel (GDN: 8 sequences x
 # 2048 tokens; Mamba-2: 16 sequences x 4096 tokens, initial and final states included); the traffic of a scan grows
 # in proportion to its tokens.
-NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.69e6 + 119.74e6) / 16384, "mamba2.scan": (788.81e6 + 671.33e6) / 65536}
+NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (291.45e6 + 120.22e6) / 16384, "mamba2.scan": (788.94e6 + 671.04e6) / 65536}
 
 
 def gdn_scan_bytes(tokens: int, s=GDN_SHAPE) -> float:
@@ -682,7 +682,30 @@ def run_sweep(args):
                                  buffer_sets=len(fns)))
                 del fns, keep
                 torch.cuda.empty_cache()
-    print(json.dumps(dict(sweep="compose_us_vs_K", timing="kernels under 100 us: 24 or more launches per CUDA-event pair "
+    # the online fold (transitions applied from the cached key / gate streams, one scan per chunk) beside the
+    # composition over materialised transitions: one request, K chunks of 1024 tokens, GDN benchmark shapes
+    fold = []
+    sg = GDN_SHAPE
+    for K in (4, 16):
+        L = 1024
+        T = K * L
+        rn = lambda *shape: torch.randn(shape, generator=gen, device="cuda")
+        kk = torch.nn.functional.normalize(rn(T, sg["H_k"], sg["d_k"]), dim=-1).to(torch.bfloat16)
+        gg = -0.1 * torch.nn.functional.softplus(rn(T, sg["H_v"]))
+        bb = torch.sigmoid(rn(T, sg["H_v"]))
+        states = rn(K, sg["H_v"], sg["d_k"], sg["d_v"])
+        cu = (np.arange(K + 1) * L).astype(np.int32)
+        ws = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+        trans = b.lkv_gdn_chunk_transition(kk, gg, bb, cu_seqlens=cu, workspace_t=ws)
+        S0 = torch.empty((sg["H_v"], sg["d_k"], sg["d_v"]), device="cuda")
+        r_fold = timer.kernel_us([lambda: b.lkv_init_state_fold(states, kk, gg, bb, cu, K, None, S0, workspace_t=ws)], 0, 7)
+        r_mat = timer.kernel_us([lambda: b.lkv_init_state(states, trans, K, b.LKV_INIT_EXACT, S0, family=b.LKV_FAMILY_GDN,
+                                                          workspace_t=ws)], 0, 7)
+        fold.append(dict(K=K, chunk_len=L, fold_us=round(r_fold["us"], 1), materialised_us=round(r_mat["us"], 1),
+                         stream_bytes=int(T * (sg["H_k"] * sg["d_k"] * 2 + 2 * sg["H_v"] * 4)),
+                         transition_bytes=int((K - 1) * sg["H_v"] * sg["d_k"] * sg["d_k"] * 4),
+                         timing="one call per event pair, L2 flushed before it"))
+    print(json.dumps(dict(sweep="compose_us_vs_K", fold_vs_materialised=fold, timing="kernels under 100 us: 24 or more launches per CUDA-event pair "
                           "inside one graph, rotating over buffer sets whose total exceeds L2, time divided by the "
                           "launches, median and p90 of 9 replays; longer ones: one launch per event pair after an L2 "
                           "flush, median and p90", rows=rows)))
@@ -776,6 +799,70 @@ def run_dry(args):
         dist.destroy_process_group()
 
 
+def run_profile_case(args):
+    """--profile-case NAME: three launches of one kernel on a small fixed case (inputs larger than L2, a few GB at most)
+    and nothing else -- the command that ncu captures for the summaries under profiles/."""
+    import torch
+
+    from paper_2608_11231_b200 import binding as b
+    torch.cuda.set_device(0)
+    b.load()
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    rn = lambda *shape: torch.randn(shape, generator=gen, device="cuda")
+    bf = torch.bfloat16
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    name = args.profile_case
+    if name == "gdn_scan":
+        s, n_seq, L = GDN_SHAPE, 8, 2048
+        T = n_seq * L
+        nrm = torch.nn.functional.normalize
+        q, k = nrm(rn(T, s["H_k"], s["d_k"]), dim=-1).to(bf), nrm(rn(T, s["H_k"], s["d_k"]), dim=-1).to(bf)
+        v, g, beta = rn(T, s["H_v"], s["d_v"]).to(bf), -0.1 * torch.nn.functional.softplus(rn(T, s["H_v"])), torch.sigmoid(rn(T, s["H_v"]))
+        S0 = rn(n_seq, s["H_v"], s["d_k"], s["d_v"])
+        o, ST = torch.empty_like(v), torch.empty_like(S0)
+        cu = (np.arange(n_seq + 1) * L).astype(np.int32)
+        fn = lambda: b.lkv_gdn_fwd(q, k, v, g, beta, S0, o, ST, cu_seqlens=cu, workspace_t=ws)
+        work = dict(tokens=T, flops=gdn_scan_flops(T))
+    elif name == "ssd_scan":
+        s, n_seq, L = SSD_SHAPE, 16, 4096
+        T = n_seq * L
+        x = rn(T, s["H"], s["P"]).to(bf)
+        dt = torch.nn.functional.softplus(-2.0 + 0.5 * rn(T, s["H"]))
+        A = -torch.exp(2.0 * torch.rand(s["H"], generator=gen, device="cuda"))
+        Bm, Cm = (rn(T, s["G"], s["N"]) / s["N"] ** 0.5).to(bf), (rn(T, s["G"], s["N"]) / s["N"] ** 0.5).to(bf)
+        S0 = rn(n_seq, s["H"], s["N"], s["P"])
+        y, ST = torch.empty_like(x), torch.empty_like(S0)
+        cu = (np.arange(n_seq + 1) * L).astype(np.int32)
+        fn = lambda: b.lkv_ssd_fwd(x, dt, A, Bm, Cm, S0, y, ST, cu_seqlens=cu, workspace_t=ws)
+        work = dict(tokens=T, flops=ssd_scan_flops(T))
+    elif name in ("gdn_compose", "mamba_compose"):
+        n_req, K = (32, 8) if name == "gdn_compose" else (32, 16)
+        if name == "gdn_compose":
+            H, dk, dv, code = GDN_SHAPE["H_v"], GDN_SHAPE["d_k"], GDN_SHAPE["d_v"], b.LKV_FAMILY_GDN
+            trans = rn(n_req * K, H, dk, dk) * (0.45 / dk ** 0.5)
+        else:
+            H, dk, dv, code = SSD_SHAPE["H"], SSD_SHAPE["N"], SSD_SHAPE["P"], b.LKV_FAMILY_MAMBA2
+            trans = -2.0 * torch.rand((n_req * K, H), generator=gen, device="cuda")
+        states = rn(n_req * K, H, dk, dv)
+        S0 = torch.empty((n_req, H, dk, dv), device="cuda")
+        ids, cu_k = np.arange(n_req * K, dtype=np.int32), (np.arange(n_req + 1) * K).astype(np.int32)
+        fn = lambda: b.lkv_init_state_batched(states, trans, ids, cu_k, n_req, b.LKV_INIT_EXACT, None, S0, family=code, workspace_t=ws)
+        nbytes = (states.numel() + S0.numel()) * 4 + (trans.numel() - (n_req * H * dk * dk if name == "gdn_compose" else 0)) * 4
+        work = dict(requests=n_req, K=K, bytes=nbytes)
+    else:
+        raise SystemExit("unknown profile case")
+    ts = []
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        ts.append(1e3 * e0.elapsed_time(e1))
+    assert b.lkv_device_status(ws) == b.LKV_OK
+    print(json.dumps(dict(profile_case=name, us_per_call=[round(t, 1) for t in ts], **work)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -785,6 +872,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true", help="composition time against K instead of the step benchmark")
     ap.add_argument("--artifacts", action="store_true", help="time of building chunk states and transitions")
+    ap.add_argument("--profile-case", default=None, choices=["gdn_scan", "ssd_scan", "gdn_compose", "mamba_compose"],
+                    help="three launches of one kernel on a small fixed case, for an ncu capture")
     ap.add_argument("--no-configs", action="store_true", help="leave the cfg1-cfg3 object out of the default line")
     ap.add_argument("--dry-run", action="store_true",
                     help="ranks on CPU over gloo with a stand-in step: exercises the launch, sharding and timing "
@@ -796,6 +885,9 @@ def main():
         sys.exit(sharding.launch_ranks(os.path.abspath(__file__), sys.argv[1:], args.gpus))
     if args.dry_run:
         run_dry(args)
+        return
+    if args.profile_case:
+        run_profile_case(args)
         return
     if args.artifacts:
         run_artifacts(args)
