@@ -95,7 +95,10 @@ extern "C" {
 #define LKV_INIT_EXACT 2 /* S_init = exact composition, Eq. 6 */
 
 /* arithmetic used for the dense contractions */
-#define LKV_COMPUTE_AUTO 0   /* tensor cores where a kernel exists for the shape, else fp32 */
+#define LKV_COMPUTE_AUTO 0   /* tensor cores where a kernel exists for the shape, else fp32.  Note: for GDN exact
+                                composition at d_k = d_v = 128 this means tf32 products (operands rounded to nearest,
+                                11-bit significands, fp32 accumulation; about 1e-3 relative on the carried part):
+                                ask for LKV_COMPUTE_FP32 where fp32 products are wanted */
 #define LKV_COMPUTE_FP32 1   /* fp32 FMA on CUDA cores everywhere (tight-tolerance / small shapes) */
 #define LKV_COMPUTE_TENSOR 2 /* tensor cores (bf16 operands in the scans, tf32 in GDN composition),
                                 fp32 accumulate; LKV_ERR_UNSUPPORTED if no such kernel fits */
