@@ -431,9 +431,19 @@ def measure_workload(name, rank, world, args, torch, b, dist, timer, peaks, with
     cold_by_size = total_input_bytes > 4 * L2_BYTES        # inputs far larger than the 126 MB L2
     steps = args.steps
 
+    fam_streams = [torch.cuda.Stream() for _ in fams[1:]]
+
     def step():
-        for f in fams:
-            f.step()
+        # the families are independent: the second one runs on a stream of its own (a fork and a join inside the
+        # step, captured into the graph like everything else), so that its CTAs fill the tail of the first one's kernels
+        cur = torch.cuda.current_stream()
+        for f, st in zip(fams[1:], fam_streams):
+            st.wait_stream(cur)
+            with torch.cuda.stream(st):
+                f.step()
+        fams[0].step()
+        for st in fam_streams:
+            cur.wait_stream(st)
 
     for _ in range(max(args.warmup, 3)):
         step()
