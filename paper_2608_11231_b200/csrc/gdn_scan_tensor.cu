@@ -81,16 +81,33 @@ struct Bars {
     // single-arrival barriers: TMA transactions and tcgen05.commit
     uint64_t full_qk[3], tiles_free_qk[3], full_v[2], g_done[2], ks_done, u_done, ds_done, o_mma_done[4], p_free[3], x_free[2];
     // 128-thread barriers (prep or mask warpgroup)
-    uint64_t m_ready[2], qs_ready[3], o_done[4], o_staged[2];
+    uint64_t m_ready[2], o_done[4], o_staged[2];
     // 64-thread barriers (the two halves of the mask warpgroup)
     uint64_t a_ready[2], p_ready[3];
     // 32-thread barriers (the scalar warp)
     uint64_t gb_ready[4];
     // 256-thread barriers (both chain warpgroups)
-    uint64_t rk_ready, uw_ready, st_ready, chain_done[4];
+    uint64_t rk_ready, uw_ready, st_ready, chain_done[4], qs_ready[3];
 };
-constexpr int kBars1 = 22, kBars128 = 11, kBars64 = 5, kBars32 = 4, kBars256 = 7;
+constexpr int kBars1 = 22, kBars128 = 8, kBars64 = 5, kBars32 = 4, kBars256 = 10;
 static_assert(sizeof(Bars) == 8 * (kBars1 + kBars128 + kBars64 + kBars32 + kBars256), "barrier table");
+
+// A quarter row of the Q tile (token tid & 63, 16-byte chunks 4 * (part & 1) .. + 3 of K-block part >> 1, part = tid >> 6)
+// multiplied in place by f.  Not inlined: the chain warps' registers are spoken for.
+static __device__ __noinline__ void scale_q_quarter(unsigned char *stage, int tid, float f) {
+    const int tq = tid & 63, part = tid >> 6;
+    unsigned char *qt = stage + (part >> 1) * (2 * kC * 128) + tq * 128;
+    const __nv_bfloat162 f2 = __float2bfloat162_rn(f);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint4 *p = reinterpret_cast<uint4 *>(qt + (((4 * (part & 1) + c) ^ (tq & 7)) << 4));
+        uint4 v = *p;
+        __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) e[i] = __hmul2(e[i], f2);
+        *p = v;
+    }
+}
 
 // Warp-level tensor-core MMA on fp16 operands (11-bit significands like tf32, but 16 k-elements per
 // instruction): acc[16 x 8] += A[16 x 16] B[16 x 8], fp32 accumulation.  Fragments as the PTX ISA lays them out.
@@ -444,16 +461,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int k = 0; k < 8; ++k)
                     umma_bf16_ts(tm + kTmKS, tm + kTmSb + 8 * k, dK + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
                 umma_commit(&bars.ks_done);
-                // (2Q) O = S^T Qs^T right behind (2K), off the chain: it reads the same bf16 state; the O columns of this
-                // parity were drained with the outputs of block b-2
-                if (has_o) {
-                    if (b >= 2) mbar_wait(&bars.o_done[(b - 2) & 3], ((b - 2) >> 2) & 1, &dead, a.status);
-                    mbar_wait(&bars.qs_ready[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        umma_bf16_ts(tm + kTmO + 64 * par, tm + kTmSb + 8 * k, dQ + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
-                }
                 // (3a) U = V^T X^T: needs the inverse of the block and the V tile (the U columns were read by (5) and (7)
                 // of the previous block, issued before)
                 mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
@@ -472,6 +479,16 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     umma_bf16_ts(tm + kTmU, tm + kTmKS + 32 * (k >> 1) + 8 * (k & 1), dX + 2 * k, idN64, has_v || k > 0);
                 umma_commit(&bars.u_done);
                 umma_commit(&bars.x_free[b & 1]);
+                // (2Q) O = S^T Qs^T while the chain warps work on U: it reads the bf16 state of this block (rewritten only after
+                // (5)), the Q tile scaled by the chain warps, and O columns that were drained with the outputs of block b-2
+                if (has_o) {
+                    if (b >= 2) mbar_wait(&bars.o_done[(b - 2) & 3], ((b - 2) >> 2) & 1, &dead, a.status);
+                    mbar_wait(&bars.qs_ready[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16_ts(tm + kTmO + 64 * par, tm + kTmSb + 8 * k, dQ + (((k >> 2) * (2 * kC * 128) + (k & 3) * 32) >> 4), idN64, k > 0);
+                }
                 // (5) accumulates onto the pre-scaled state; B = K tile read MN-major (rows = tokens)
                 mbar_wait(&bars.uw_ready, par, &dead, a.status);
                 tc_fence_after_sync();
@@ -596,24 +613,6 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             }
             fence_async_smem();
             mbar_arrive(&bars.m_ready[b & 1]);
-            // ---- Q tile of block b scaled in place by scale gam_t ((1) has read it: its result was masked before the
-            // inverse began): thread = (token, 64-column half)
-            if (has_o) {
-                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);   // this thread reads what the TMA wrote
-                unsigned char *qt = sm + (b % kQKStages) * kQKStage + (x >> 6) * (2 * kC * 128) + (x & 63) * 128;
-                const __nv_bfloat162 f2 = __float2bfloat162_rn(a.scale * sc[2 * kC + (x & 63)]);
-#pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
-                    uint4 *p = reinterpret_cast<uint4 *>(qt + ((c ^ (x & 7)) << 4));
-                    uint4 v = *p;
-                    __nv_bfloat162 *e = reinterpret_cast<__nv_bfloat162 *>(&v);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) e[i] = __hmul2(e[i], f2);
-                    *p = v;
-                }
-                fence_async_smem();
-                mbar_arrive(&bars.qs_ready[b % kQKStages]);
-            }
         }
     } else if (warp >= 8) {
         // ======================================================= mask warpgroup: epilogue of (1) and Q scaling, as far ahead of the
@@ -807,6 +806,15 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tmem_st_wait();
             tc_fence_before_sync();
             mbar_arrive(&bars.rk_ready);
+            // While (3b) is on its way: the Q tile of block b scaled in place by scale gam_t for (2Q).  (1) has read the tile
+            // once the block's inverse is ready (the mask epilogue came before it); thread = (token, quarter of the row).
+            if (has_o) {
+                mbar_wait(&bars.m_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+                mbar_wait(&bars.full_qk[b % kQKStages], (b / kQKStages) & 1, &dead, a.status);   // this thread reads what the TMA wrote
+                scale_q_quarter(sm + (b % kQKStages) * kQKStage, tid, a.scale * sc[2 * kC + (tid & 63)]);
+                fence_async_smem();
+                mbar_arrive(&bars.qs_ready[b % kQKStages]);
+            }
             // u_t[j], tokens 32*half..+31 -> Uw = w o u as bf16 pairs over the first 16 of this thread's own 32 columns, u over the rest
             mbar_wait(&bars.u_done, par, &dead, a.status);
             tc_fence_after_sync();
