@@ -117,6 +117,10 @@ __device__ __forceinline__ void mma_f16_16x8x16(float (&acc)[4], const uint32_t 
         : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ uint32_t pack_bf16_early(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     const __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const uint32_t *>(&v);
@@ -140,6 +144,18 @@ __device__ __forceinline__ void store_acc(float *p, const float (&acc)[4], float
     *reinterpret_cast<float2 *>(p + (gid + 8) * kLd + 2 * tig) = make_float2(sgn * acc[2], sgn * acc[3]);
 }
 
+// Byte offset of element (row m, column i) of a bf16 operand tile with 128-byte rows and the 128-byte swizzle
+__device__ __forceinline__ uint32_t x_offset(int m, int i) { return m * 128u + ((((uint32_t)i >> 3) ^ (m & 7u)) << 4) + (i & 7) * 2u; }
+// Final entries of M also go, times beta of their column and rounded to bf16, into the operand X = M diag(beta) of the
+// block's triangular solve: no second pass over M.  Accumulator tile [16 x 8] at (m0, i0):
+__device__ __forceinline__ void store_acc_x(unsigned char *xb, const float *beta, int m0, int i0, const float (&acc)[4], float sgn,
+                                            int gid, int tig) {
+    const int i = i0 + 2 * tig;
+    const float b0 = sgn * beta[i], b1 = sgn * beta[i + 1];
+    *reinterpret_cast<uint32_t *>(xb + x_offset(m0 + gid, i)) = pack_bf16_early(acc[0] * b0, acc[1] * b1);
+    *reinterpret_cast<uint32_t *>(xb + x_offset(m0 + gid + 8, i)) = pack_bf16_early(acc[2] * b0, acc[3] * b1);
+}
+
 // The inverse M = (I + A)^{-1} of the unit lower triangular 64x64 matrix of a block is built by doubling:
 // 8x8 diagonal blocks by forward substitution, then three merges
 //     inv [[L1, 0], [A21, L2]] = [[inv L1, 0], [-inv(L2) A21 inv(L1), inv L2]]
@@ -149,7 +165,7 @@ __device__ __forceinline__ void store_acc(float *p, const float (&acc)[4], float
 //
 // 16 -> 32: half (8 columns from 8 nh) of the 16x16 block (c + 1, c): X = A_rc M_cc, M_rc = -M_rr X; X passes
 // through the unused block (c, r) above the diagonal to change from accumulator to operand layout.
-__device__ __forceinline__ void inv_merge32(const float *Af, float *Mf, int c, int nh, int gid, int tig) {
+__device__ __forceinline__ void inv_merge32(const float *Af, float *Mf, unsigned char *xb, const float *beta, int c, int nh, int gid, int tig) {
     const int r = c + 1;
     uint32_t a[4], b0, b1;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -165,6 +181,7 @@ __device__ __forceinline__ void inv_merge32(const float *Af, float *Mf, int c, i
     frag_b(b0, b1, xs, gid, tig);
     mma_f16_16x8x16(acc, a, b0, b1);
     store_acc(Mf + (16 * r) * kLd + 16 * c + 8 * nh, acc, -1.f, gid, tig);
+    store_acc_x(xb, beta, 16 * r, 16 * c + 8 * nh, acc, -1.f, gid, tig);
 }
 // 32 -> 64, first half: T = A21 inv(L1) with A21 = A[32.., 0..31], inv(L1) = M[0..31, 0..31] (lower triangular by 16x16
 // blocks).  Warp (mt, nb) computes rows 16 mt .. +15, columns 16 nb .. +15 of T into the scratch M[0..31, 32..63].
@@ -196,7 +213,7 @@ __device__ __forceinline__ void inv_merge64_a(const float *Af, float *Mf, int mt
     }
 }
 // 32 -> 64, second half: M[32.., 0..31] = -inv(L2) T with inv(L2) = M[32.., 32..] (lower triangular by blocks).
-__device__ __forceinline__ void inv_merge64_b(float *Mf, int mt, int nb, int gid, int tig) {
+__device__ __forceinline__ void inv_merge64_b(float *Mf, unsigned char *xb, const float *beta, int mt, int nb, int gid, int tig) {
     float acc[2][2][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt)
@@ -220,7 +237,7 @@ __device__ __forceinline__ void inv_merge64_b(float *Mf, int mt, int nb, int gid
     for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[nt][0][i] += acc[nt][1][i];
-        store_acc(Mf + (32 + 16 * mt) * kLd + 16 * nb + 8 * nt, acc[nt][0], -1.f, gid, tig);
+        store_acc_x(xb, beta, 32 + 16 * mt, 16 * nb + 8 * nt, acc[nt][0], -1.f, gid, tig);   // nobody reads these entries of M again
     }
 }
 __device__ __forceinline__ void named_bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
@@ -515,11 +532,18 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
         // ======================================================= prep warpgroup: the inverse and its operand, ahead of the chain
         const int x = tid - 384;                 // 0..127
         float *Mf = reinterpret_cast<float *>(sm + kOffM);
+        // both X buffers start as zeros: only entries on or below the block diagonal are ever written
+        for (int e = x; e < 2 * kC * 128 / 16; e += 128) reinterpret_cast<uint4 *>(sm + kOffX)[e] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll 1
         for (int b = 0; b < nblk; ++b) {
             const float *sc = gb + (b & 3) * kGbFloats;
+            const float *beta = sc + kC;
             // ---- A comes from the mask warpgroup (epilogue of (1))
             mbar_wait(&bars.a_ready[b & 1], (b >> 1) & 1, &dead, a.status);
+            // X = M diag(beta) (bf16) is written as the entries of M become final; the buffer of this parity was read by
+            // (3b) of block b-2
+            if (b >= 2) mbar_wait(&bars.x_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
+            unsigned char *xb = sm + kOffX + (b & 1) * (kC * 128);
             named_bar_sync(1, 128);   // every thread is done with the fp32 M of the previous block
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
             // ---- M = (I + A)^{-1} by doubling.  8x8 diagonal blocks: thread (k, c) solves column c of block k by forward
@@ -548,6 +572,10 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
 #pragma unroll
                 for (int t = 0; t < 8; ++t) Mf[(8 * k + t) * kLd + 8 * k + c] = xv[t];
+                const float bc = beta[8 * k + c];
+#pragma unroll
+                for (int t = 0; t < 8; ++t)
+                    *reinterpret_cast<__nv_bfloat16 *>(xb + x_offset(8 * k + t, 8 * k + c)) = __float2bfloat16_rn(xv[t] * bc);
             }
             named_bar_sync(1, 128);
             // 8 -> 16 in fp32: thread = (16-block k, row i, column pair) of the 8x8 block below the diagonal;
@@ -575,6 +603,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                     m1 = fmaf(dv, ts[m * kLd + j0 + 1], m1);
                 }
                 *reinterpret_cast<float2 *>(Mf + (16 * k + 8 + i) * kLd + 16 * k + j0) = make_float2(-m0, -m1);
+                *reinterpret_cast<uint32_t *>(xb + x_offset(16 * k + 8 + i, 16 * k + j0)) =
+                    pack_bf16(-m0 * beta[16 * k + j0], -m1 * beta[16 * k + j0 + 1]);
                 // the 8x8 block above the diagonal of the 16x16 block reads as part of the operands later: zero
                 *reinterpret_cast<float2 *>(Mf + (16 * k + i) * kLd + 16 * k + 8 + j0) = make_float2(0.f, 0.f);
             }
@@ -582,34 +612,12 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             {
                 const int wq = warp & 3, gid = lane >> 2, tig = lane & 3;
                 // 16 -> 32: blocks (1, 0) and (3, 2), one half block per warp
-                inv_merge32(Af, Mf, 2 * (wq >> 1), wq & 1, gid, tig);
+                inv_merge32(Af, Mf, xb, beta, 2 * (wq >> 1), wq & 1, gid, tig);
                 named_bar_sync(1, 128);
                 // 32 -> 64: one 16x16 block of the 32x32 result per warp
                 inv_merge64_a(Af, Mf, wq >> 1, wq & 1, gid, tig);
                 named_bar_sync(1, 128);
-                inv_merge64_b(Mf, wq >> 1, wq & 1, gid, tig);
-                named_bar_sync(1, 128);
-            }
-            // ---- X = M diag(beta) as bf16 operand (zeros above the block diagonal); the buffer of this parity was
-            // read by (3b) of block b-2
-            if (b >= 2) mbar_wait(&bars.x_free[b & 1], ((b - 2) >> 1) & 1, &dead, a.status);
-            unsigned char *xb = sm + kOffX + (b & 1) * (kC * 128);
-            {
-                // thread = (row m, half of the columns)
-                const int m = x & 63, q0 = 2 * (x >> 6);
-#pragma unroll 1
-                for (int q = q0; q < q0 + 2; ++q) {
-                    float v[16];
-                    const bool live = q <= (m >> 4);
-#pragma unroll
-                    for (int c = 0; c < 16; c += 4) {
-                        const int i = 16 * q + c;
-                        const float4 mv = live ? *reinterpret_cast<const float4 *>(Mf + m * kLd + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        const float4 be = *reinterpret_cast<const float4 *>(sc + kC + i);
-                        v[c] = mv.x * be.x; v[c + 1] = mv.y * be.y; v[c + 2] = mv.z * be.z; v[c + 3] = mv.w * be.w;
-                    }
-                    store_row_chunks(xb, m, 2 * q, v);
-                }
+                inv_merge64_b(Mf, xb, beta, wq >> 1, wq & 1, gid, tig);
             }
             fence_async_smem();
             mbar_arrive(&bars.m_ready[b & 1]);
