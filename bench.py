@@ -205,6 +205,15 @@ class Family:
             self.full_out = torch.empty((tokens, s["H"], s["P"]), dtype=bf, device="cuda")
         self.full_tokens = tokens
 
+    def full_prefill_segmented(self):
+        """The same full prefill with the sequence cut into segments scanned in parallel (GDN; the library picks the count)."""
+        b, d = self.b, self.full
+        if getattr(self, "seg_scratch", None) is None:
+            s = GDN_SHAPE
+            self.seg_scratch = self.torch.empty(64 * s["H_v"] * s["d_k"] * s["d_v"] * 4, dtype=self.torch.uint8, device="cuda")
+        b.lkv_gdn_fwd_segmented(d["q"], d["k"], d["v"], d["g"], d["beta"], None, self.full_out, self.full_ST, n_segments=0,
+                                scratch=self.seg_scratch, workspace_t=self.ws_scan)
+
     def full_prefill(self):
         b, d = self.b, self.full
         if self.fam == "gdn":
@@ -503,6 +512,13 @@ def measure_workload(name, rank, world, args, torch, b, dist, timer, peaks, with
             t_cached = 1e-3 * (parts[f"{f.fam}.init_exact"]["us"] + parts[f"{f.fam}.scan"]["us"]) / f.n_req
             full[f.fam] = dict(tokens=f.full_tokens, us=1e3 * t, tokens_per_s=f.full_tokens / (t * 1e-3),
                                cached_path_us_per_request=1e3 * t_cached, cached_over_full=t_cached / t)
+            if f.fam == "gdn":
+                # the same prefill as a sequence-parallel scan (lkv_gdn_fwd_segmented, segment count chosen by the library)
+                g2 = timer.graph_of(f.full_prefill_segmented)
+                t2 = 1e-3 * statistics.median(1e3 * x for x in timer.flushed(g2.replay, max(steps, 5)))
+                full[f.fam]["segmented_us"] = 1e3 * t2
+                full[f.fam]["segments"] = max(1, min((148 // GDN_SHAPE["H_v"] + 3) // 2, f.full_tokens // 512))
+                f.seg_scratch = None
             del f.full, f.full_out
 
     detail = {}

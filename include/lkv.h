@@ -279,6 +279,26 @@ int lkv_gdn_fwd(const void *q, const void *k, const void *v, const float *g, con
                 const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream);
 
 /*
+ * lkv_gdn_fwd for ONE long sequence, cut into n_segments segments that are scanned in parallel (a sequence-parallel
+ * prefill; Eq. 5 and Eq. 6 applied inside one request): pass 1 computes, in one launch, the state each of the first
+ * n_segments - 1 segments reaches from an empty start (the first one from S0) and the accumulated transitions of
+ * segments 1 .. n_segments - 2; pass 2 composes the state every segment starts from (exact composition); pass 3 scans
+ * all segments at once from those states.  About twice the arithmetic of lkv_gdn_fwd, but n_segments times the
+ * CTAs: for a single sequence on an otherwise idle GPU it shortens the chain of dependent blocks.
+ * Same arguments and results as lkv_gdn_fwd (results equal up to the rounding of the composition, which uses the
+ * arithmetic of d->compute: tf32 products under AUTO / TENSOR at d = 128); requires d->n_seq == 1, d_k == d_v,
+ * state_dtype fp32.  scratch: device, 16-byte aligned, >= lkv_gdn_segmented_scratch_bytes(d, n_segments) bytes, owned by
+ * the caller.  n_segments == 1 is lkv_gdn_fwd itself; n_segments == 0 lets the library choose (as many segments as keep
+ * both scanning passes within one round of CTAs on the current GPU, none shorter than 512 tokens; the scratch-size call
+ * makes the same choice).  Five stream operations besides the three kernel launches
+ * (memsets / device copies of single states).  (The paper has no counterpart: its prefill is the plain scan.)
+ */
+int lkv_gdn_fwd_segmented(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                          const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, int n_segments,
+                          void *scratch, size_t scratch_bytes, void *stream);
+size_t lkv_gdn_segmented_scratch_bytes(const lkv_gdn_desc *d, int n_segments);
+
+/*
  * Mamba-2 (SSD) scan from an initial state (Eq. 1 with Eq. 2; Algorithm 1, line 3).
  * For each sequence and head, in token order:
  *     S_t = exp(dt_t A_h) S_{t-1} + dt_t B_t x_t^T,      y_t = S_t^T C_t

@@ -28,7 +28,8 @@ LKV_COMPUTE_AUTO, LKV_COMPUTE_FP32, LKV_COMPUTE_TENSOR = 0, 1, 2
 LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
-           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_init_state_fold", "lkv_state_rel_error",
+           "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_init_state_fold", "lkv_gdn_fwd_segmented",
+           "lkv_gdn_segmented_scratch_bytes", "lkv_state_rel_error",
            "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_device_status_static",
            "lkv_selftest_bounded_wait", "lkv_status_string", "lkv_version")
 
@@ -82,6 +83,10 @@ def load() -> ctypes.CDLL:
         lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_init_state_fold.argtypes = [vp, vp, vp, vp, vp, ci, vp, ctypes.POINTER(lkv_init_desc), ci, ci, vp]
         lib.lkv_init_state_fold.restype = ci
+        lib.lkv_gdn_fwd_segmented.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), ci, vp, ctypes.c_size_t, vp]
+        lib.lkv_gdn_fwd_segmented.restype = ci
+        lib.lkv_gdn_segmented_scratch_bytes.argtypes = [ctypes.POINTER(lkv_gdn_desc), ci]
+        lib.lkv_gdn_segmented_scratch_bytes.restype = ctypes.c_size_t
         lib.lkv_state_rel_error.argtypes = [vp, vp, vp, ci, ctypes.c_size_t, vp, ctypes.c_size_t, vp]
         lib.lkv_state_rel_error_workspace_bytes.argtypes = [ci, ctypes.c_size_t]
         lib.lkv_state_rel_error_workspace_bytes.restype = ctypes.c_size_t
@@ -267,6 +272,31 @@ def lkv_gdn_fwd(q, k, v, g, beta, S0=None, o=None, S_T=None, *, cu_seqlens=None,
                             ctypes.byref(d), _stream(stream))
     if st != LKV_OK:
         raise LkvError(st, "lkv_gdn_fwd")
+    return o, S_T
+
+
+def lkv_gdn_fwd_segmented(q, k, v, g, beta, S0=None, o=None, S_T=None, *, n_segments: int, scale: float = 0.0,
+                          compute: int = LKV_COMPUTE_AUTO, scratch: Optional[torch.Tensor] = None,
+                          workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """lkv_gdn_fwd for one long sequence, its n_segments segments scanned in parallel (states and transitions of the
+    segments, exact composition, then all segments at once).  S0: [1, H_v, d, d] fp32 or None.  Returns (o, S_T)."""
+    T, H_k, d_k = q.shape
+    _, H_v, d_v = v.shape
+    d = lkv_gdn_desc(T_total=T, n_seq=1, cu_seqlens=None, H_k=H_k, H_v=H_v, d_k=d_k, d_v=d_v, io_dtype=_dtype_code(v),
+                     compute=compute, scale=float(scale), state_dtype=0, workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(v.device, lkv_workspace_bytes(LKV_WS_GDN, d, 2 * n_segments))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    need = int(load().lkv_gdn_segmented_scratch_bytes(ctypes.byref(d), int(n_segments)))
+    if scratch is None:
+        scratch = torch.empty(max(need, 16), dtype=torch.uint8, device=v.device)
+    if o is None:
+        o = torch.empty_like(v)
+    if S_T is None:
+        S_T = torch.empty((1, H_v, d_k, d_v), dtype=torch.float32, device=v.device)
+    st = load().lkv_gdn_fwd_segmented(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(S0), _ptr(o), _ptr(S_T),
+                                      ctypes.byref(d), int(n_segments), _ptr(scratch), scratch.numel(), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_gdn_fwd_segmented")
     return o, S_T
 
 

@@ -75,6 +75,10 @@ struct GdnArgs {
     float scale;
     int32_t s0_identity;         // start every sequence from S = I (d_k == d_v) instead of S0; with v == nullptr (read
                                  // as zeros) the final state is then the sequence's accumulated transition; o may be nullptr
+    // Sequences tr_first .. n_seq-1 are "transition sequences": they run in that mode (S = I, v = 0, no outputs) whatever
+    // the call's own mode is, over the token range of sequence (seq - tr_first + tr_src0).  cu has n_ranges + 1 entries
+    // (the ranges of sequences 0 .. tr_first-1); a plain call has n_ranges = tr_first = n_seq.
+    int32_t n_ranges, tr_first, tr_src0;
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1], then the launch order: sequence of grid row y at [n_seq + 1 + y]
 };

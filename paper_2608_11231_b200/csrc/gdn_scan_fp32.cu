@@ -37,19 +37,21 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
     float *bs = cg + kC;                   // [kC]
     float *gs = bs + kC;                   // [kC]
 
-    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
+    const int h = blockIdx.x, seq = a.cu[a.n_ranges + 1 + blockIdx.y];   // launch order: longest sequence first
+    const bool tr = seq >= a.tr_first;                                    // transition sequence
+    const int rg = tr ? seq - a.tr_first + a.tr_src0 : seq;
     const int hk = h / (a.H_v / a.H_k);
     const int tid = threadIdx.x;
     const int j = tid % DV, tg = tid / DV;
-    const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
+    const int t_begin = a.cu[rg], t_end = a.cu[rg + 1];
     const T *q = static_cast<const T *>(a.q);
     const T *k = static_cast<const T *>(a.k);
-    const T *v = static_cast<const T *>(a.v);
-    T *o = static_cast<T *>(a.o);
+    const T *v = tr ? nullptr : static_cast<const T *>(a.v);
+    T *o = tr ? nullptr : static_cast<T *>(a.o);
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * dk * DV;
 
     for (int idx = tid; idx < dk * DV; idx += 256)
-        S[idx] = a.s0_identity ? (idx / DV == idx % DV ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + idx] : 0.f);
+        S[idx] = (a.s0_identity || tr) ? (idx / DV == idx % DV ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + idx] : 0.f);
 
     for (int t0 = t_begin; t0 < t_end; t0 += kC) {
         const int n = min(kC, t_end - t0);

@@ -305,18 +305,21 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     __shared__ volatile int dead;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int h = blockIdx.x, seq = a.cu[a.n_seq + 1 + blockIdx.y];   // launch order: longest sequence first
+    const int h = blockIdx.x, seq = a.cu[a.n_ranges + 1 + blockIdx.y];   // launch order: longest sequence first
+    const bool tr = seq >= a.tr_first;                                    // transition sequence
+    const int rg = tr ? seq - a.tr_first + a.tr_src0 : seq;
+    const bool s0_id = a.s0_identity || tr;
     const int hk = h / (a.H_v / a.H_k);
-    const int t_begin = a.cu[seq], t_end = a.cu[seq + 1];
+    const int t_begin = a.cu[rg], t_end = a.cu[rg + 1];
     const int nblk = (t_end - t_begin + kC - 1) / kC;
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * kD * kD;
-    const bool has_v = a.v != nullptr, has_o = a.o != nullptr;
+    const bool has_v = a.v != nullptr && !tr, has_o = a.o != nullptr && !tr;
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
-        if (a.S_T && (a.S_T != a.S0 || a.s0_identity || a.S_add))
+        if (a.S_T && (a.S_T != a.S0 || s0_id || a.S_add))
             for (int e = tid; e < kD * kD; e += kThreads)
                 store_state(a.S_T, a.st_bf16, sbase + e,
-                            (a.s0_identity ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f)) +
+                            (s0_id ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f)) +
                                 (a.S_add ? a.S_add[sbase + e] : 0.f));
         return;
     }
@@ -771,7 +774,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const int m = 64 * half + 16 * q + c;
-                    v[c] = a.s0_identity ? (m == j ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + static_cast<size_t>(m) * kD + j] : 0.f);
+                    v[c] = s0_id ? (m == j ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + static_cast<size_t>(m) * kD + j] : 0.f);
                     rr[c] = __float_as_uint(v[c] * gamC);
                 }
                 tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr);

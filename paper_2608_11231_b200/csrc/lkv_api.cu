@@ -209,7 +209,9 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
 
 // lkv_gdn_fwd, and with `transition` set the scan from S = I with v = 0 whose final state is the chunk transition
 // what: 0 = scan, 1 = chunk transitions (start from S = I, v read as zeros), 2 = one step of the online fold (v read as
-// zeros, S_add added to the final state)
+// zeros, S_add added to the final state), 3 = local states and transitions in one launch: d->n_seq = 2 m - 1 sequences,
+// the first m of them scans over the m ranges of d->cu_seqlens (m + 1 entries), the other m - 1 the transitions of ranges
+// 1 .. m-1 (the kernels' "transition sequences")
 static int gdn_impl(const void *q, const void *k, const void *v, const float *g, const float *beta,
                     const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream, int what,
                     const float *S_add = nullptr) {
@@ -220,10 +222,11 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     if (st_bf16 && S_T && S_T == S0) return LKV_ERR_OVERLAP;   // an fp32 input cannot be a bf16 output
     if (d->H_k < 1 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1 || d->H_v % d->H_k != 0) return LKV_ERR_DIM;
     std::vector<int32_t> cu;
-    int st = check_seqs(d->T_total, d->n_seq, d->cu_seqlens, cu);
+    const int n_ranges = what == 3 ? (d->n_seq + 1) / 2 : d->n_seq;
+    int st = check_seqs(d->T_total, n_ranges, d->cu_seqlens, cu);
     if (st != LKV_OK) return st;
     if (d->n_seq == 0) return LKV_OK;
-    if (transition && d->d_k != d->d_v) return LKV_ERR_DIM;
+    if ((transition || what == 3) && d->d_k != d->d_v) return LKV_ERR_DIM;
     if (d->T_total > 0 && (!q || !k || !g || !beta)) return LKV_ERR_NULL;
     if (what == 0 && d->T_total > 0 && !v) return LKV_ERR_NULL;
     if (!o && !S_T) return LKV_ERR_NULL;   // nothing to compute
@@ -253,6 +256,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     a.n_seq = d->n_seq; a.T_total = d->T_total; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
     a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
     a.s0_identity = transition ? 1 : 0;
+    a.n_ranges = n_ranges; a.tr_first = n_ranges; a.tr_src0 = what == 3 ? 1 : 0;
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
     const bool tensor_fits = gdn_scan_tensor_supported(a, io_bf16);
@@ -269,7 +273,16 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         use_tensor = tensor_fits;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    append_launch_order(cu, d->n_seq);
+    if (what == 3) {
+        // launch order over all 2 m - 1 sequences, longest first; transition sequence j runs over range j - m + 1
+        std::vector<int32_t> order(d->n_seq);
+        auto len = [&](int sq) { const int r = sq < n_ranges ? sq : sq - n_ranges + 1; return cu[r + 1] - cu[r]; };
+        for (int i = 0; i < d->n_seq; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return len(x) > len(y); });
+        cu.insert(cu.end(), order.begin(), order.end());
+    } else {
+        append_launch_order(cu, d->n_seq);
+    }
     st = place_indices(a.cu, cu, d->workspace, s);
     if (st != LKV_OK) return st;
     const cudaError_t e = use_tensor ? launch_gdn_scan_tensor(a, s) : launch_gdn_scan_fp32(a, io_bf16, s);
@@ -328,6 +341,93 @@ int lkv_init_state_fold(const void *states, const void *k, const float *g, const
                       static_cast<const float *>(states) + static_cast<size_t>(c) * state_elems);
         if (st != LKV_OK) return st;
     }
+    return LKV_OK;
+}
+
+// n_segments == 0: as many segments as keep both scanning passes within one round of CTAs on this GPU -- (2 n - 3) H_v and
+// n H_v CTAs, one per SM -- and no segment shorter than 512 tokens
+static int auto_segments(const lkv_gdn_desc *d) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        sms = 148;
+    }
+    int n = (sms / (d->H_v > 0 ? d->H_v : 1) + 3) / 2;
+    if (n > d->T_total / 512) n = d->T_total / 512;
+    return n < 1 ? 1 : n;
+}
+
+size_t lkv_gdn_segmented_scratch_bytes(const lkv_gdn_desc *d, int n_segments) {
+    if (!d || n_segments < 0 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1) return 0;
+    if (n_segments == 0) n_segments = auto_segments(d);
+    if (n_segments < 2) return 0;
+    return sizeof(float) * static_cast<size_t>(4 * n_segments - 3) * d->H_v * d->d_k * d->d_v;
+}
+
+int lkv_gdn_fwd_segmented(const void *q, const void *k, const void *v, const float *g, const float *beta,
+                          const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, int n_segments,
+                          void *scratch, size_t scratch_bytes, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (n_segments < 0) return LKV_ERR_DIM;
+    if (n_segments == 0) {
+        if (d->H_v < 1 || d->T_total < 0) return LKV_ERR_DIM;
+        n_segments = auto_segments(d);
+    }
+    if (n_segments == 1) return lkv_gdn_fwd(q, k, v, g, beta, S0, o, S_T, d, stream);
+    if (d->n_seq != 1 || d->state_dtype != LKV_DTYPE_F32) return LKV_ERR_UNSUPPORTED;   // one sequence, fp32 final state
+    if (d->d_k != d->d_v) return LKV_ERR_DIM;                                            // transitions are d_k x d_k
+    if (d->T_total < 0) return LKV_ERR_DIM;
+    if (d->cu_seqlens && (d->cu_seqlens[0] != 0 || d->cu_seqlens[1] != d->T_total)) return LKV_ERR_INDEX;
+    if (!scratch || scratch_bytes < lkv_gdn_segmented_scratch_bytes(d, n_segments)) return LKV_ERR_WORKSPACE;
+    if (!aligned16(scratch)) return LKV_ERR_ALIGN;
+    if (!o && !S_T) return LKV_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n_seg = n_segments, n_st = n_seg - 1;
+    const size_t slot = static_cast<size_t>(d->H_v) * d->d_k * d->d_v;   // floats per state of all heads
+    float *pool = static_cast<float *>(scratch);                        // S_local of segments 0 .. n_st-1, then T of 1 .. n_st-1
+    float *trans = pool + (static_cast<size_t>(n_st) - 1) * slot;       // T of segment j at trans + j slots (slot 0 is never read)
+    float *S_init = pool + (2 * static_cast<size_t>(n_st) - 1) * slot;  // [n_seg]
+    float *S_fin = S_init + static_cast<size_t>(n_seg) * slot;          // [n_seg]; first the initial states of pass 1
+    // segment boundaries on multiples of 64 tokens, so that every block of the segmented scan is a block of the plain one
+    const int per = ((d->T_total + n_seg - 1) / n_seg + 63) / 64 * 64;
+    std::vector<int32_t> bounds(n_seg + 1);
+    for (int i = 0; i <= n_seg; ++i) bounds[i] = std::min<long long>(static_cast<long long>(i) * per, d->T_total);
+    // ---- pass 1: local states of segments 0 .. n_st-1 (segment 0 from S0) and transitions of segments 1 .. n_st-1, one launch
+    if (cudaMemsetAsync(S_fin, 0, sizeof(float) * slot * n_st, s) != cudaSuccess) return LKV_ERR_CUDA;
+    if (S0 && cudaMemcpyAsync(S_fin, S0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LKV_ERR_CUDA;
+    lkv_gdn_desc d1 = *d;
+    d1.n_seq = 2 * n_st - 1;
+    d1.T_total = bounds[n_st];
+    d1.cu_seqlens = bounds.data();
+    int st = gdn_impl(q, k, v, g, beta, S_fin, nullptr, pool, &d1, stream, 3);
+    if (st != LKV_OK) return st;
+    // ---- pass 2: the state each segment starts from, by exact composition (Eq. 6) over the segments before it
+    if (S0) {
+        if (cudaMemcpyAsync(S_init, S0, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s) != cudaSuccess) return LKV_ERR_CUDA;
+    } else if (cudaMemsetAsync(S_init, 0, sizeof(float) * slot, s) != cudaSuccess) {
+        return LKV_ERR_CUDA;
+    }
+    {
+        std::vector<int32_t> ids, cu_k(n_st + 1, 0);
+        for (int r = 0; r < n_st; ++r) {
+            for (int j = 0; j <= r; ++j) ids.push_back(j);
+            cu_k[r + 1] = static_cast<int32_t>(ids.size());
+        }
+        lkv_init_desc di{};
+        di.family = LKV_FAMILY_GDN; di.H = d->H_v; di.d_k = d->d_k; di.d_v = d->d_v; di.n_chunks = n_st;
+        di.state_dtype = LKV_DTYPE_F32; di.sel_index = 0; di.compute = d->compute; di.chunk_ids = nullptr;
+        di.workspace = d->workspace; di.workspace_bytes = d->workspace_bytes;
+        st = lkv_init_state_batched(pool, trans, ids.data(), cu_k.data(), n_st, LKV_INIT_EXACT, nullptr, S_init + slot, &di, stream);
+        if (st != LKV_OK) return st;
+    }
+    // ---- pass 3: every segment scanned from its initial state, all at once
+    lkv_gdn_desc d3 = *d;
+    d3.n_seq = n_seg;
+    d3.cu_seqlens = bounds.data();
+    st = gdn_impl(q, k, v, g, beta, S_init, o, S_fin, &d3, stream, 0);
+    if (st != LKV_OK) return st;
+    if (S_T && cudaMemcpyAsync(S_T, S_fin + static_cast<size_t>(n_seg - 1) * slot, sizeof(float) * slot, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return LKV_ERR_CUDA;
     return LKV_OK;
 }
 

@@ -245,3 +245,23 @@ def test_fold_argument_errors(lib):
     assert call(gd(), cu_p=bad.ctypes.data) == b.LKV_ERR_INDEX
     ids[1] = 3
     assert call(gd()) == b.LKV_ERR_INDEX
+
+
+def test_segmented_prefill_argument_errors(lib):
+    f = lambda d, n=3, scratch=fake(9), nbytes=1 << 30, S_T=fake(8): lib.lkv_gdn_fwd_segmented(
+        fake(1), fake(2), fake(3), fake(4), fake(5), None, fake(7), S_T, ctypes.byref(d) if d is not None else None, n,
+        scratch, nbytes, None)
+    lib.lkv_gdn_fwd_segmented.argtypes = [ctypes.c_void_p] * 8 + [ctypes.POINTER(b.lkv_gdn_desc), ctypes.c_int, ctypes.c_void_p,
+                                          ctypes.c_size_t, ctypes.c_void_p]
+    assert f(None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(), n=-1) == b.LKV_ERR_DIM
+    cu = np.array([0, 60, 100], dtype=np.int32)
+    assert f(_gdn_desc(n_seq=2, cu_seqlens=cu.ctypes.data)) == b.LKV_ERR_UNSUPPORTED     # one sequence only
+    assert f(_gdn_desc(state_dtype=b.LKV_DTYPE_BF16)) == b.LKV_ERR_UNSUPPORTED
+    assert f(_gdn_desc(d_k=64, d_v=32)) == b.LKV_ERR_DIM
+    assert f(_gdn_desc(), scratch=None) == b.LKV_ERR_WORKSPACE
+    assert f(_gdn_desc(), nbytes=1024) == b.LKV_ERR_WORKSPACE
+    assert f(_gdn_desc(), scratch=fake(9) + 4) == b.LKV_ERR_ALIGN
+    need = lib.lkv_gdn_segmented_scratch_bytes(ctypes.byref(_gdn_desc()), 3)
+    assert need == (4 * 3 - 3) * 4 * 64 * 64 * 4
+    assert lib.lkv_gdn_segmented_scratch_bytes(ctypes.byref(_gdn_desc()), 1) == 0

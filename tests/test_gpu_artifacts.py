@@ -213,3 +213,31 @@ def test_final_states_stored_as_bf16_are_the_rounded_fp32_ones():
     # a bf16 pool built this way feeds the initialisers
     S_last = b.lkv_init_state(S16, None, 3, b.LKV_INIT_LAST, family=b.LKV_FAMILY_MAMBA2)
     assert torch.equal(S_last, S16[2].float())
+
+
+@pytest.mark.parametrize("case", [dict(T=1000, n=3, d=128, io="bf16", compute="auto", tol=TOL_BF16),
+                                  dict(T=700, n=4, d=128, io="bf16", compute="auto", tol=TOL_BF16),
+                                  dict(T=130, n=2, d=128, io="bf16", compute="auto", tol=TOL_BF16),
+                                  dict(T=50, n=3, d=128, io="bf16", compute="auto", tol=TOL_BF16),
+                                  dict(T=500, n=3, d=64, io="f32", compute="fp32", tol=TOL_F32)])
+def test_segmented_prefill_equals_the_plain_scan_and_the_oracle(case):
+    """One sequence cut into segments scanned in parallel (states and transitions of the segments, exact composition,
+    all segments at once) == the plain scan == the oracle's token recurrence."""
+    import torch
+    rng = np.random.default_rng(43 + case["T"])
+    T, d, H_k, H_v = case["T"], case["d"], 2, 4
+    tok = wl.gdn_tokens(rng, T, H_k, H_v, d, d, io=case["io"], live_chunk_len=256)
+    S0 = rng.standard_normal((1, H_v, d, d)).astype(np.float32)
+    dt = torch.bfloat16 if case["io"] == "bf16" else None
+    compute = b.LKV_COMPUTE_AUTO if case["compute"] == "auto" else b.LKV_COMPUTE_FP32
+    args = (dev(tok["q"], dt), dev(tok["k"], dt), dev(tok["v"], dt), dev(tok["g"]), dev(tok["beta"]))
+    o_ref, ST_ref = oracle.gdn_seq(tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], S0[0])
+    for s0 in (S0, None):
+        o, ST = b.lkv_gdn_fwd_segmented(*args, None if s0 is None else dev(s0), n_segments=case["n"], compute=compute)
+        o_p, ST_p = b.lkv_gdn_fwd(*args, None if s0 is None else dev(s0), compute=compute)
+        assert maxrel(host(o), host(o_p)) <= case["tol"] and maxrel(host(ST), host(ST_p)) <= case["tol"]
+        if s0 is not None:
+            assert maxrel(host(o), o_ref) <= case["tol"] and maxrel(host(ST)[0], ST_ref) <= case["tol"]
+    # the first segment is the same blocks from the same state: its outputs are the plain scan's, bit for bit
+    per = ((T + case["n"] - 1) // case["n"] + 63) // 64 * 64
+    assert torch.equal(o[:per], o_p[:per])
