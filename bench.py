@@ -80,6 +80,7 @@ class Family:
         rng = np.random.default_rng(seed)
         self.n_req = len(reqs)
         shared = any(r.get("shared_pool") for r in reqs)
+        self.shared = shared
         ks = [r["K"] for r in reqs]
         self.cu_k = np.concatenate([[0], np.cumsum(ks)]).astype(np.int32)
         if shared:
@@ -150,6 +151,32 @@ class Family:
             setattr(c, n, getattr(self, n).clone())
         c.ws_init, c.ws_scan = self.ws_init.clone(), self.ws_scan.clone()
         return c
+
+    def micro_batches(self, m):
+        """The same requests as m instances over slices of this one's buffers (every request has its own pool entries and
+        tokens, contiguous in request order): the end-to-end step pipelines them, so that the results of one micro-batch
+        travel to the host while the inputs of the next travel to the device."""
+        import copy
+        if self.shared or self.n_req < m:
+            return [self]
+        out = []
+        per_tok = ("q", "k", "v", "g", "beta", "x", "B", "C", "dt")
+        for i in range(m):
+            r0, r1 = self.n_req * i // m, self.n_req * (i + 1) // m
+            p0, p1, t0, t1 = int(self.cu_k[r0]), int(self.cu_k[r1]), int(self.cu_seq[r0]), int(self.cu_seq[r1])
+            c = copy.copy(self)
+            c.n_req = r1 - r0
+            c.cu_k, c.cu_seq = self.cu_k[r0:r1 + 1] - p0, self.cu_seq[r0:r1 + 1] - t0
+            c.ids = np.arange(p1 - p0, dtype=np.int32)
+            cut = lambda n, t: t[p0:p1] if n in ("states", "trans") else t[t0:t1] if n in per_tok else t
+            c.host = {n: cut(n, t) for n, t in self.host.items()}
+            c.dev = {n: cut(n, t) for n, t in self.dev.items()}
+            for n in ("S0_last", "S0", "S_T", "host_S_T"):
+                setattr(c, n, getattr(self, n)[r0:r1])
+            c.out, c.host_out = self.out[t0:t1], self.host_out[t0:t1]
+            c.ws_init, c.ws_scan = self.ws_init.clone(), self.ws_scan.clone()
+            out.append(c)
+        return out
 
     def upload(self):
         for n, t in self.host.items():
@@ -484,12 +511,14 @@ def measure_workload(name, rank, world, args, torch, b, dist, timer, peaks, with
 
     ms_e2e, e2e_steps = None, 0
     if with_e2e:
-        e2e_streams = [torch.cuda.Stream() for _ in fams]
+        # the requests of a step are independent: they go through in micro-batches (four per family), one stream each, so
+        # that the device->host copies of one overlap the host->device copies of the next
+        e2e_units = [u for f in fams for u in f.micro_batches(4)]
+        e2e_streams = [torch.cuda.Stream() for _ in e2e_units]
 
         def step_e2e():
-            # one stream per family: the device->host copies of one overlap the host->device copies of the other
             cur = torch.cuda.current_stream()
-            for f, st in zip(fams, e2e_streams):
+            for f, st in zip(e2e_units, e2e_streams):
                 st.wait_stream(cur)
                 with torch.cuda.stream(st):
                     f.upload()
