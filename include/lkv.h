@@ -299,6 +299,25 @@ int lkv_gdn_fwd_segmented(const void *q, const void *k, const void *v, const flo
 size_t lkv_gdn_segmented_scratch_bytes(const lkv_gdn_desc *d, int n_segments);
 
 /*
+ * Host-resident cache -> device staging pool (Section 4.1, "Environment": the cached artefacts live in host memory and
+ * are loaded at serving time).  The chunks that a batch of requests names are copied, each once, from pools in HOST
+ * memory (pinned for asynchronous copies) into compact pools in device memory, and the requests' chunk ids are rewritten
+ * to the slots of the staging pools, ready for lkv_init_state_batched with d->n_chunks = *n_staged.
+ *
+ *   host_states, host_transitions  HOST pools laid out as lkv_init_desc describes (n_chunks = d->n_chunks entries);
+ *                                  host_transitions may be NULL (single-state modes), then dev_transitions must be too
+ *   chunk_ids                      HOST int32[n_ids], ids into the host pools, in any order, repeats allowed
+ *   dev_states, dev_transitions    device staging pools with room for `capacity` chunks
+ *   staged_ids                     HOST out int32[n_ids]: slot of chunk_ids[i]; slots are given in order of first appearance
+ *   n_staged                       HOST out: number of distinct chunks copied
+ * One cudaMemcpyAsync per chunk and pool on `stream`; nothing is copied when an argument is wrong or the distinct chunks
+ * exceed `capacity` (LKV_ERR_WORKSPACE).  The host pools must stay valid until the copies have run.
+ */
+int lkv_stage_chunks(const void *host_states, const void *host_transitions, const int32_t *chunk_ids, int n_ids,
+                     void *dev_states, void *dev_transitions, int capacity, int32_t *staged_ids, int32_t *n_staged,
+                     const lkv_init_desc *d, void *stream);
+
+/*
  * Mamba-2 (SSD) scan from an initial state (Eq. 1 with Eq. 2; Algorithm 1, line 3).
  * For each sequence and head, in token order:
  *     S_t = exp(dt_t A_h) S_{t-1} + dt_t B_t x_t^T,      y_t = S_t^T C_t

@@ -29,7 +29,7 @@ LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
            "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_init_state_fold", "lkv_gdn_fwd_segmented",
-           "lkv_gdn_segmented_scratch_bytes", "lkv_state_rel_error",
+           "lkv_gdn_segmented_scratch_bytes", "lkv_stage_chunks", "lkv_state_rel_error",
            "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_device_status_static",
            "lkv_selftest_bounded_wait", "lkv_status_string", "lkv_version")
 
@@ -83,6 +83,8 @@ def load() -> ctypes.CDLL:
         lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_init_state_fold.argtypes = [vp, vp, vp, vp, vp, ci, vp, ctypes.POINTER(lkv_init_desc), ci, ci, vp]
         lib.lkv_init_state_fold.restype = ci
+        lib.lkv_stage_chunks.argtypes = [vp, vp, vp, ci, vp, vp, ci, vp, vp, ctypes.POINTER(lkv_init_desc), vp]
+        lib.lkv_stage_chunks.restype = ci
         lib.lkv_gdn_fwd_segmented.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), ci, vp, ctypes.c_size_t, vp]
         lib.lkv_gdn_fwd_segmented.restype = ci
         lib.lkv_gdn_segmented_scratch_bytes.argtypes = [ctypes.POINTER(lkv_gdn_desc), ci]
@@ -345,6 +347,24 @@ def lkv_init_state_fold(states: torch.Tensor, k, g, beta, cu_tokens, K: int, chu
     if st != LKV_OK:
         raise LkvError(st, "lkv_init_state_fold")
     return S0
+
+
+def lkv_stage_chunks(host_states: torch.Tensor, host_transitions: Optional[torch.Tensor], chunk_ids, dev_states: torch.Tensor,
+                     dev_transitions: Optional[torch.Tensor], *, family: int, stream=None):
+    """Copies the distinct chunks named by chunk_ids from host pools (pinned CPU tensors) into the device staging pools.
+    Returns (staged_ids int32 numpy array for lkv_init_state_batched, number of chunks copied)."""
+    ids = _host_i32(chunk_ids)
+    n, H, d_k, d_v = host_states.shape
+    d = lkv_init_desc(family=family, H=H, d_k=d_k, d_v=d_v, n_chunks=n, state_dtype=_dtype_code(host_states), sel_index=0,
+                      compute=LKV_COMPUTE_AUTO, chunk_ids=None, workspace=None, workspace_bytes=0)
+    staged = np.empty(ids.size, dtype=np.int32)
+    n_staged = ctypes.c_int32(0)
+    st = load().lkv_stage_chunks(host_states.data_ptr(), None if host_transitions is None else host_transitions.data_ptr(),
+                                 _hp(ids), ids.size, _ptr(dev_states), _ptr(dev_transitions), int(dev_states.shape[0]),
+                                 staged.ctypes.data, ctypes.addressof(n_staged), ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_stage_chunks")
+    return staged, int(n_staged.value)
 
 
 def lkv_gdn_chunk_transition(k, g, beta, transitions=None, *, cu_seqlens=None, H_v: Optional[int] = None,

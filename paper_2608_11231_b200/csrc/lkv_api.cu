@@ -431,6 +431,49 @@ int lkv_gdn_fwd_segmented(const void *q, const void *k, const void *v, const flo
     return LKV_OK;
 }
 
+int lkv_stage_chunks(const void *host_states, const void *host_transitions, const int32_t *chunk_ids, int n_ids,
+                     void *dev_states, void *dev_transitions, int capacity, int32_t *staged_ids, int32_t *n_staged,
+                     const lkv_init_desc *d, void *stream) {
+    int st = check_init_desc(d);
+    if (st != LKV_OK) return st;
+    if (n_ids < 0 || capacity < 0) return LKV_ERR_DIM;
+    if (!n_staged) return LKV_ERR_NULL;
+    *n_staged = 0;
+    if (n_ids == 0) return LKV_OK;
+    if (!host_states || !dev_states || !chunk_ids || !staged_ids) return LKV_ERR_NULL;
+    if ((host_transitions == nullptr) != (dev_transitions == nullptr)) return LKV_ERR_NULL;   // both pools or neither
+    if (!aligned16(dev_states) || !aligned16(dev_transitions)) return LKV_ERR_ALIGN;
+    // slots in order of first appearance; everything is checked before the first copy is queued
+    std::vector<int32_t> slot_of(d->n_chunks, -1), order;
+    for (int i = 0; i < n_ids; ++i) {
+        const int32_t c = chunk_ids[i];
+        if (c < 0 || c >= d->n_chunks) return LKV_ERR_INDEX;
+        if (slot_of[c] < 0) {
+            slot_of[c] = static_cast<int32_t>(order.size());
+            order.push_back(c);
+        }
+    }
+    if (static_cast<long long>(order.size()) > capacity) return LKV_ERR_WORKSPACE;
+    const size_t es = d->state_dtype == LKV_DTYPE_BF16 ? 2 : 4;
+    const size_t state_b = es * static_cast<size_t>(d->H) * d->d_k * d->d_v;
+    const size_t trans_b = sizeof(float) * static_cast<size_t>(d->H) * (d->family == LKV_FAMILY_GDN ? static_cast<size_t>(d->d_k) * d->d_k : 1);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (size_t k = 0; k < order.size(); ++k) {
+        const size_t c = static_cast<size_t>(order[k]);
+        if (cudaMemcpyAsync(static_cast<char *>(dev_states) + k * state_b, static_cast<const char *>(host_states) + c * state_b,
+                            state_b, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            (host_transitions &&
+             cudaMemcpyAsync(static_cast<char *>(dev_transitions) + k * trans_b, static_cast<const char *>(host_transitions) + c * trans_b,
+                             trans_b, cudaMemcpyHostToDevice, s) != cudaSuccess)) {
+            cudaGetLastError();
+            return LKV_ERR_CUDA;
+        }
+    }
+    for (int i = 0; i < n_ids; ++i) staged_ids[i] = slot_of[chunk_ids[i]];
+    *n_staged = static_cast<int32_t>(order.size());
+    return LKV_OK;
+}
+
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream) {
     if (!d) return LKV_ERR_NULL;
     if (d->H < 1) return LKV_ERR_DIM;

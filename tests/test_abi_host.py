@@ -265,3 +265,25 @@ def test_segmented_prefill_argument_errors(lib):
     need = lib.lkv_gdn_segmented_scratch_bytes(ctypes.byref(_gdn_desc()), 3)
     assert need == (4 * 3 - 3) * 4 * 64 * 64 * 4
     assert lib.lkv_gdn_segmented_scratch_bytes(ctypes.byref(_gdn_desc()), 1) == 0
+
+
+def test_stage_chunks_argument_errors(lib):
+    lib.lkv_stage_chunks.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.POINTER(b.lkv_init_desc), ctypes.c_void_p]
+    ids = np.array([3, 1, 3, 0], dtype=np.int32)
+    out = np.zeros(4, dtype=np.int32)
+    n = ctypes.c_int32(-1)
+
+    def call(d, idp=ids.ctypes.data, n_ids=4, hs=fake(1), ht=fake(2), ds=fake(3), dt=fake(4), cap=8, outp=out.ctypes.data,
+             np_=ctypes.addressof(n)):
+        return lib.lkv_stage_chunks(hs, ht, idp, n_ids, ds, dt, cap, outp, np_, ctypes.byref(d) if d is not None else None, None)
+    assert call(None) == b.LKV_ERR_NULL
+    assert call(_desc(), n_ids=-1) == b.LKV_ERR_DIM
+    assert call(_desc(), np_=None) == b.LKV_ERR_NULL
+    assert call(_desc(), n_ids=0) == b.LKV_OK and n.value == 0            # nothing named, nothing copied
+    assert call(_desc(), hs=None) == b.LKV_ERR_NULL
+    assert call(_desc(), ht=None) == b.LKV_ERR_NULL                       # one transition pool without the other
+    assert call(_desc(), ds=fake(3) + 8) == b.LKV_ERR_ALIGN
+    assert call(_desc(n_chunks=3)) == b.LKV_ERR_INDEX                     # id 3 of a 3-chunk pool
+    assert call(_desc(), cap=2) == b.LKV_ERR_WORKSPACE                    # three distinct chunks, room for two

@@ -241,3 +241,37 @@ def test_segmented_prefill_equals_the_plain_scan_and_the_oracle(case):
     # the first segment is the same blocks from the same state: its outputs are the plain scan's, bit for bit
     per = ((T + case["n"] - 1) // case["n"] + 63) // 64 * 64
     assert torch.equal(o[:per], o_p[:per])
+
+
+@pytest.mark.parametrize("family", ["gdn", "mamba2"])
+def test_staging_from_a_host_pool_feeds_the_initialisers(family):
+    """The cache lives in (pinned) host memory; the chunks a batch names are staged once each into a compact device pool
+    and the ids rewritten: composing from the staged pool == composing from the whole pool on the device, bit for bit."""
+    import torch
+    rng = np.random.default_rng(44)
+    n, H = 40, 3
+    if family == "gdn":
+        code, dk, dv = b.LKV_FAMILY_GDN, 128, 128
+        trans = wl.synthetic_gdn_transitions(rng, n, H, dk)
+    else:
+        code, dk, dv = b.LKV_FAMILY_MAMBA2, 128, 64
+        trans = wl.synthetic_logdecay(rng, n, H)
+    states = wl.synthetic_states(rng, n, H, dk, dv)
+    h_states, h_trans = torch.from_numpy(states).pin_memory(), torch.from_numpy(trans).pin_memory()
+    n_req, K = 6, 5
+    ids = rng.integers(0, n, size=n_req * K).astype(np.int32)     # repeats across and inside requests
+    cu_k = (np.arange(n_req + 1) * K).astype(np.int32)
+    distinct = len(set(ids.tolist()))
+    d_states = torch.empty((distinct,) + states.shape[1:], device="cuda")
+    d_trans = torch.empty((distinct,) + trans.shape[1:], device="cuda")
+    staged, n_staged = b.lkv_stage_chunks(h_states, h_trans, ids, d_states, d_trans, family=code)
+    assert n_staged == distinct and staged.max() == distinct - 1
+    torch.cuda.synchronize()
+    for slot, c in {int(s): int(c) for s, c in zip(staged, ids)}.items():
+        assert torch.equal(d_states[slot].cpu(), h_states[c]) and torch.equal(d_trans[slot].cpu(), h_trans[c])
+    got = b.lkv_init_state_batched(d_states, d_trans, staged, cu_k, n_req, b.LKV_INIT_EXACT, family=code)
+    ref = b.lkv_init_state_batched(dev(states), dev(trans), ids, cu_k, n_req, b.LKV_INIT_EXACT, family=code)
+    assert torch.equal(got, ref)
+    with pytest.raises(b.LkvError) as e:       # a staging pool that is too small is refused before anything is copied
+        b.lkv_stage_chunks(h_states, h_trans, ids, d_states[: distinct - 1], d_trans[: distinct - 1], family=code)
+    assert e.value.status == b.LKV_ERR_WORKSPACE
