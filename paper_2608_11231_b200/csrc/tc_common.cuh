@@ -1,6 +1,6 @@
 // Blackwell (sm_100a) building blocks used by the tensor-core kernels: mbarriers with bounded
 // waits, TMA tile loads, TMEM allocation, tcgen05 MMA issue / commit and TMEM <-> register moves.
-// Everything here is single-CTA (cta_group::1); no cluster multicast is used anywhere.
+// Everything here is single-CTA (cta_group::1): no instruction here addresses more than one CTA of a cluster.
 #pragma once
 
 #include <cuda.h>
