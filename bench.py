@@ -800,6 +800,8 @@ def run_artifacts(args):
     calls = {
         "gdn_states": lambda: b.lkv_gdn_fwd(q, k, v, g, beta, None, None, st_g, cu_seqlens=cu, want_outputs=False, workspace_t=ws),
         "gdn_transitions": lambda: b.lkv_gdn_chunk_transition(k, g, beta, tr_g, cu_seqlens=cu, workspace_t=ws),
+        "gdn_states_and_transitions_one_launch": lambda: b.lkv_gdn_chunk_artifacts(k, v, g, beta, st_g, tr_g, cu_seqlens=cu,
+                                                                                   workspace_t=ws),
         "mamba_states": lambda: b.lkv_ssd_fwd(x, dt, A, Bm, Cm, None, None, st_m, cu_seqlens=cu, want_outputs=False, workspace_t=ws),
         "mamba_logdecays": lambda: b.lkv_mamba_chunk_logdecay(dt, A, lam, cu_seqlens=cu, workspace_t=ws),
     }

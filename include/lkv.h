@@ -351,6 +351,18 @@ int lkv_gdn_chunk_transition(const void *k, const float *g, const float *beta, f
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream);
 
 /*
+ * Both cached artefacts of every GDN chunk in ONE launch: states[c] = the state chunk c reaches from an empty start
+ * (S_local) and transitions[c] = its accumulated transition T_C (Eq. 5), fp32 [n_seq, H_v, d, d] each, the chunks being
+ * the sequences of d->cu_seqlens.  Every chunk is scanned twice inside the launch (once with its values from S = 0, once
+ * with v = 0 from S = I); what one launch buys over lkv_gdn_fwd + lkv_gdn_chunk_transition is that the two scans of a
+ * chunk run side by side, which matters when a few chunks do not fill the GPU.  Results are bit-identical to those two
+ * calls.  k, v, g, beta and errors as for lkv_gdn_fwd (d_k == d_v required; state_dtype must be fp32); the workspace must
+ * be sized for 2 * n_seq sequences (lkv_workspace_bytes(LKV_WS_GDN, d, 2 * n_seq, 0)).
+ */
+int lkv_gdn_chunk_artifacts(const void *k, const void *v, const float *g, const float *beta, float *states,
+                            float *transitions, const lkv_gdn_desc *d, void *stream);
+
+/*
  * GDN exact composition for ONE request WITHOUT materialised transitions (the "online fold": Eq. 6 evaluated as the
  * chain of Eq. 5 with every T_C applied token by token from the chunk's cached key / gate stream):
  *     S <- S_{c_1};   S <- (scan of chunk c_j's tokens with v = 0 from S) + S_{c_j},   j = 2..K.

@@ -29,7 +29,7 @@ LKV_WS_INIT, LKV_WS_GDN, LKV_WS_SSD = 0, 1, 2
 
 EXPORTS = ("lkv_init_state", "lkv_init_state_batched", "lkv_init_state_batched_static", "lkv_gdn_fwd", "lkv_ssd_fwd",
            "lkv_gdn_chunk_transition", "lkv_mamba_chunk_logdecay", "lkv_init_state_fold", "lkv_gdn_fwd_segmented",
-           "lkv_gdn_segmented_scratch_bytes", "lkv_stage_chunks", "lkv_state_rel_error",
+           "lkv_gdn_segmented_scratch_bytes", "lkv_stage_chunks", "lkv_gdn_chunk_artifacts", "lkv_state_rel_error",
            "lkv_state_rel_error_workspace_bytes", "lkv_workspace_bytes", "lkv_device_status", "lkv_device_status_static",
            "lkv_selftest_bounded_wait", "lkv_status_string", "lkv_version")
 
@@ -83,6 +83,8 @@ def load() -> ctypes.CDLL:
         lib.lkv_mamba_chunk_logdecay.argtypes = [vp] * 3 + [ctypes.POINTER(lkv_ssd_desc), vp]
         lib.lkv_init_state_fold.argtypes = [vp, vp, vp, vp, vp, ci, vp, ctypes.POINTER(lkv_init_desc), ci, ci, vp]
         lib.lkv_init_state_fold.restype = ci
+        lib.lkv_gdn_chunk_artifacts.argtypes = [vp] * 6 + [ctypes.POINTER(lkv_gdn_desc), vp]
+        lib.lkv_gdn_chunk_artifacts.restype = ci
         lib.lkv_stage_chunks.argtypes = [vp, vp, vp, ci, vp, vp, ci, vp, vp, ctypes.POINTER(lkv_init_desc), vp]
         lib.lkv_stage_chunks.restype = ci
         lib.lkv_gdn_fwd_segmented.argtypes = [vp] * 8 + [ctypes.POINTER(lkv_gdn_desc), ci, vp, ctypes.c_size_t, vp]
@@ -388,6 +390,30 @@ def lkv_gdn_chunk_transition(k, g, beta, transitions=None, *, cu_seqlens=None, H
     if st != LKV_OK:
         raise LkvError(st, "lkv_gdn_chunk_transition")
     return transitions
+
+
+def lkv_gdn_chunk_artifacts(k, v, g, beta, states=None, transitions=None, *, cu_seqlens=None,
+                            compute: int = LKV_COMPUTE_AUTO, workspace_t: Optional[torch.Tensor] = None, stream=None):
+    """S_local and T_C of every chunk (sequence of cu_seqlens) in one launch.  Returns (states, transitions),
+    fp32 [n_seq, H_v, d, d] each."""
+    T, H_k, d_k = k.shape
+    _, H_v, d_v = v.shape
+    cu = _host_i32(cu_seqlens)
+    n_seq = 1 if cu is None else cu.size - 1
+    d = lkv_gdn_desc(T_total=T, n_seq=n_seq, cu_seqlens=None if cu is None else cu.ctypes.data, H_k=H_k, H_v=H_v,
+                     d_k=d_k, d_v=d_v, io_dtype=_dtype_code(k), compute=compute, scale=0.0, state_dtype=0,
+                     workspace=None, workspace_bytes=0)
+    ws_t = workspace_t if workspace_t is not None else workspace(k.device, lkv_workspace_bytes(LKV_WS_GDN, d, 2 * n_seq))
+    d.workspace, d.workspace_bytes = ws_t.data_ptr(), ws_t.numel()
+    if states is None:
+        states = torch.empty((n_seq, H_v, d_k, d_v), dtype=torch.float32, device=k.device)
+    if transitions is None:
+        transitions = torch.empty((n_seq, H_v, d_k, d_k), dtype=torch.float32, device=k.device)
+    st = load().lkv_gdn_chunk_artifacts(_ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(states), _ptr(transitions),
+                                        ctypes.byref(d), _stream(stream))
+    if st != LKV_OK:
+        raise LkvError(st, "lkv_gdn_chunk_artifacts")
+    return states, transitions
 
 
 def lkv_mamba_chunk_logdecay(dt, A, logdecay=None, *, cu_seqlens=None, workspace_t: Optional[torch.Tensor] = None,

@@ -79,6 +79,7 @@ struct GdnArgs {
     // the call's own mode is, over the token range of sequence (seq - tr_first + tr_src0).  cu has n_ranges + 1 entries
     // (the ranges of sequences 0 .. tr_first-1); a plain call has n_ranges = tr_first = n_seq.
     int32_t n_ranges, tr_first, tr_src0;
+    float *tr_out;               // where transition sequence tr_first + i stores its final state (index i), or nullptr: S_T like the others
     int32_t *status;
     IndexBlock<kScanIdxCap> cu;  // cu_seqlens[n_seq + 1], then the launch order: sequence of grid row y at [n_seq + 1 + y]
 };

@@ -49,6 +49,8 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
     const T *v = tr ? nullptr : static_cast<const T *>(a.v);
     T *o = tr ? nullptr : static_cast<T *>(a.o);
     const size_t sbase = (static_cast<size_t>(seq) * a.H_v + h) * dk * DV;
+    float *ST = (tr && a.tr_out) ? a.tr_out : a.S_T;   // final state of this sequence
+    const size_t obase = (tr && a.tr_out) ? (static_cast<size_t>(seq - a.tr_first) * a.H_v + h) * dk * DV : sbase;
 
     for (int idx = tid; idx < dk * DV; idx += 256)
         S[idx] = (a.s0_identity || tr) ? (idx / DV == idx % DV ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + idx] : 0.f);
@@ -151,10 +153,10 @@ __global__ void __launch_bounds__(256) gdn_scan_fp32_kernel(const __grid_constan
         }
         __syncthreads();
     }
-    if (a.S_T) {
+    if (ST) {
         __syncthreads();
         for (int idx = tid; idx < dk * DV; idx += 256)
-            store_state(a.S_T, a.st_bf16, sbase + idx, S[idx] + (a.S_add ? a.S_add[sbase + idx] : 0.f));
+            store_state(ST, a.st_bf16, obase + idx, S[idx] + (a.S_add ? a.S_add[sbase + idx] : 0.f));
     }
 }
 

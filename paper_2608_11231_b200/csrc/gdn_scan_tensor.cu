@@ -316,9 +316,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
     const bool has_v = a.v != nullptr && !tr, has_o = a.o != nullptr && !tr;
 
     if (nblk == 0) {  // empty sequence: hand the state through untouched
-        if (a.S_T && (a.S_T != a.S0 || s0_id || a.S_add))
+        float *ST = (tr && a.tr_out) ? a.tr_out : a.S_T;   // final state of this sequence
+        const size_t obase = (tr && a.tr_out) ? (static_cast<size_t>(seq - a.tr_first) * a.H_v + h) * kD * kD : sbase;
+        if (ST && (ST != a.S0 || s0_id || a.S_add))
             for (int e = tid; e < kD * kD; e += kThreads)
-                store_state(a.S_T, a.st_bf16, sbase + e,
+                store_state(ST, a.st_bf16, obase + e,
                             (s0_id ? (e / kD == e % kD ? 1.f : 0.f) : (a.S0 ? a.S0[sbase + e] : 0.f)) +
                                 (a.S_add ? a.S_add[sbase + e] : 0.f));
         return;
@@ -867,7 +869,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_wait(&bars.ds_done, par, &dead, a.status);
             tc_fence_after_sync();
             if (last) {
-                if (a.S_T && !dead) {
+                // where this sequence's final state goes: a transition sequence may have a buffer of its own
+                const bool own = seq >= a.tr_first && a.tr_out != nullptr;
+                float *ST = own ? a.tr_out : a.S_T;
+                const size_t obase = own ? (static_cast<size_t>(seq - a.tr_first) * a.H_v + h) * kD * kD : sbase;
+                if (ST && !dead) {
 #pragma unroll 1
                     for (int q = 0; q < 4; ++q) {
                         uint32_t rr[16];
@@ -875,8 +881,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                         tmem_ld_wait();
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
-                            const size_t e = sbase + static_cast<size_t>(64 * half + 16 * q + c) * kD + j;
-                            store_state(a.S_T, a.st_bf16, e, __uint_as_float(rr[c]) + (a.S_add ? a.S_add[e] : 0.f));
+                            const size_t e = static_cast<size_t>(64 * half + 16 * q + c) * kD + j;
+                            store_state(ST, a.st_bf16, obase + e, __uint_as_float(rr[c]) + (a.S_add ? a.S_add[sbase + e] : 0.f));
                         }
                     }
                 }

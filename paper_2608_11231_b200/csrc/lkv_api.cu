@@ -212,9 +212,11 @@ int lkv_init_state_batched(const void *states, const void *transitions, const in
 // zeros, S_add added to the final state), 3 = local states and transitions in one launch: d->n_seq = 2 m - 1 sequences,
 // the first m of them scans over the m ranges of d->cu_seqlens (m + 1 entries), the other m - 1 the transitions of ranges
 // 1 .. m-1 (the kernels' "transition sequences")
+// 4 = local states and transitions of every sequence in one launch: d->n_seq = 2 m sequences over the m ranges of
+// d->cu_seqlens, the last m of them transition sequences that write to tr_out
 static int gdn_impl(const void *q, const void *k, const void *v, const float *g, const float *beta,
                     const float *S0, void *o, void *S_T, const lkv_gdn_desc *d, void *stream, int what,
-                    const float *S_add = nullptr) {
+                    const float *S_add = nullptr, float *tr_out = nullptr) {
     const bool transition = what == 1;
     if (!d) return LKV_ERR_NULL;
     if (!dtype_ok(d->io_dtype) || !compute_ok(d->compute) || !dtype_ok(d->state_dtype)) return LKV_ERR_MODE;
@@ -222,11 +224,11 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     if (st_bf16 && S_T && S_T == S0) return LKV_ERR_OVERLAP;   // an fp32 input cannot be a bf16 output
     if (d->H_k < 1 || d->H_v < 1 || d->d_k < 1 || d->d_v < 1 || d->H_v % d->H_k != 0) return LKV_ERR_DIM;
     std::vector<int32_t> cu;
-    const int n_ranges = what == 3 ? (d->n_seq + 1) / 2 : d->n_seq;
+    const int n_ranges = what == 3 ? (d->n_seq + 1) / 2 : what == 4 ? d->n_seq / 2 : d->n_seq;
     int st = check_seqs(d->T_total, n_ranges, d->cu_seqlens, cu);
     if (st != LKV_OK) return st;
     if (d->n_seq == 0) return LKV_OK;
-    if ((transition || what == 3) && d->d_k != d->d_v) return LKV_ERR_DIM;
+    if ((transition || what >= 3) && d->d_k != d->d_v) return LKV_ERR_DIM;
     if (d->T_total > 0 && (!q || !k || !g || !beta)) return LKV_ERR_NULL;
     if (what == 0 && d->T_total > 0 && !v) return LKV_ERR_NULL;
     if (!o && !S_T) return LKV_ERR_NULL;   // nothing to compute
@@ -239,7 +241,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         // outputs may not overlap inputs (S_T == S0 exactly is the one allowed alias) nor each other
         const size_t es = d->io_dtype == LKV_DTYPE_BF16 ? 2 : 4, T = static_cast<size_t>(d->T_total);
         const size_t qk_b = es * T * d->H_k * d->d_k, v_b = es * T * d->H_v * d->d_v, gb_b = sizeof(float) * T * d->H_v;
-        const size_t st_in = sizeof(float) * static_cast<size_t>(d->n_seq) * d->H_v * d->d_k * d->d_v;
+        const size_t st_in = sizeof(float) * static_cast<size_t>(what == 4 ? n_ranges : d->n_seq) * d->H_v * d->d_k * d->d_v;
         const size_t st_b = st_bf16 ? st_in / 2 : st_in;
         const void *in[6] = {q, k, v, g, beta, S0};
         const size_t in_b[6] = {qk_b, qk_b, v ? v_b : 0, gb_b, gb_b, S0 ? st_in : 0};
@@ -256,7 +258,7 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
     a.n_seq = d->n_seq; a.T_total = d->T_total; a.H_k = d->H_k; a.H_v = d->H_v; a.d_k = d->d_k; a.d_v = d->d_v;
     a.scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf(static_cast<float>(d->d_k));
     a.s0_identity = transition ? 1 : 0;
-    a.n_ranges = n_ranges; a.tr_first = n_ranges; a.tr_src0 = what == 3 ? 1 : 0;
+    a.n_ranges = n_ranges; a.tr_first = n_ranges; a.tr_src0 = what == 3 ? 1 : 0; a.tr_out = tr_out;
     a.status = static_cast<int32_t *>(d->workspace);
     const bool io_bf16 = d->io_dtype == LKV_DTYPE_BF16;
     const bool tensor_fits = gdn_scan_tensor_supported(a, io_bf16);
@@ -273,10 +275,10 @@ static int gdn_impl(const void *q, const void *k, const void *v, const float *g,
         use_tensor = tensor_fits;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (what == 3) {
-        // launch order over all 2 m - 1 sequences, longest first; transition sequence j runs over range j - m + 1
+    if (what >= 3) {
+        // launch order over all sequences, longest first; transition sequence j runs over range j - m + (1 or 0)
         std::vector<int32_t> order(d->n_seq);
-        auto len = [&](int sq) { const int r = sq < n_ranges ? sq : sq - n_ranges + 1; return cu[r + 1] - cu[r]; };
+        auto len = [&](int sq) { const int r = sq < n_ranges ? sq : sq - n_ranges + (what == 3 ? 1 : 0); return cu[r + 1] - cu[r]; };
         for (int i = 0; i < d->n_seq; ++i) order[i] = i;
         std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return len(x) > len(y); });
         cu.insert(cu.end(), order.begin(), order.end());
@@ -472,6 +474,23 @@ int lkv_stage_chunks(const void *host_states, const void *host_transitions, cons
     for (int i = 0; i < n_ids; ++i) staged_ids[i] = slot_of[chunk_ids[i]];
     *n_staged = static_cast<int32_t>(order.size());
     return LKV_OK;
+}
+
+int lkv_gdn_chunk_artifacts(const void *k, const void *v, const float *g, const float *beta, float *states,
+                            float *transitions, const lkv_gdn_desc *d, void *stream) {
+    if (!d) return LKV_ERR_NULL;
+    if (d->state_dtype != LKV_DTYPE_F32) return LKV_ERR_MODE;
+    if (d->n_seq > 0 && (!states || !transitions)) return LKV_ERR_NULL;
+    if (d->n_seq < 0 || d->n_seq > (1 << 29)) return LKV_ERR_DIM;
+    if (!aligned16(transitions)) return LKV_ERR_ALIGN;
+    {
+        const size_t st_b = sizeof(float) * static_cast<size_t>(d->n_seq > 0 ? d->n_seq : 0) * d->H_v * d->d_k * d->d_v;
+        if (overlaps(states, st_b, transitions, st_b)) return LKV_ERR_OVERLAP;
+    }
+    lkv_gdn_desc d2 = *d;
+    d2.n_seq = 2 * d->n_seq;   // every chunk twice: once as a scan from the empty state, once as a transition sequence
+    // q is not needed for the states: the key tensor stands in for it (its read-outs are not written)
+    return gdn_impl(k, k, v, g, beta, nullptr, nullptr, states, &d2, stream, 4, nullptr, transitions);
 }
 
 int lkv_mamba_chunk_logdecay(const float *dt, const float *A, float *logdecay, const lkv_ssd_desc *d, void *stream) {

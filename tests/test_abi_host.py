@@ -287,3 +287,17 @@ def test_stage_chunks_argument_errors(lib):
     assert call(_desc(), ds=fake(3) + 8) == b.LKV_ERR_ALIGN
     assert call(_desc(n_chunks=3)) == b.LKV_ERR_INDEX                     # id 3 of a 3-chunk pool
     assert call(_desc(), cap=2) == b.LKV_ERR_WORKSPACE                    # three distinct chunks, room for two
+
+
+def test_chunk_artifacts_argument_errors(lib):
+    lib.lkv_gdn_chunk_artifacts.argtypes = [ctypes.c_void_p] * 6 + [ctypes.POINTER(b.lkv_gdn_desc), ctypes.c_void_p]
+    f = lambda d, st=fake(6), tr=fake(7): lib.lkv_gdn_chunk_artifacts(fake(2), fake(3), fake(4), fake(5), st, tr,
+                                                                       ctypes.byref(d) if d is not None else None, None)
+    assert f(None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(), st=None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(), tr=None) == b.LKV_ERR_NULL
+    assert f(_gdn_desc(state_dtype=b.LKV_DTYPE_BF16)) == b.LKV_ERR_MODE
+    assert f(_gdn_desc(d_k=64, d_v=32)) == b.LKV_ERR_DIM
+    assert f(_gdn_desc(), tr=fake(6) + 1024) == b.LKV_ERR_OVERLAP            # transitions inside the states buffer
+    assert f(_gdn_desc(), tr=fake(7) + 4) == b.LKV_ERR_ALIGN
+    assert f(_gdn_desc(workspace_bytes=8)) == b.LKV_ERR_WORKSPACE

@@ -275,3 +275,19 @@ def test_staging_from_a_host_pool_feeds_the_initialisers(family):
     with pytest.raises(b.LkvError) as e:       # a staging pool that is too small is refused before anything is copied
         b.lkv_stage_chunks(h_states, h_trans, ids, d_states[: distinct - 1], d_trans[: distinct - 1], family=code)
     assert e.value.status == b.LKV_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("compute", [b.LKV_COMPUTE_AUTO, b.LKV_COMPUTE_FP32])
+def test_one_launch_producer_equals_the_two_calls_bit_for_bit(compute):
+    import torch
+    rng = np.random.default_rng(45)
+    lens = [200, 64, 0, 131, 77, 1024]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    tok = wl.gdn_tokens(rng, int(cu[-1]), 2, 4, 128, 128, io="bf16", live_chunk_len=128)
+    bf = torch.bfloat16
+    k, v, g, beta = dev(tok["k"], bf), dev(tok["v"], bf), dev(tok["g"]), dev(tok["beta"])
+    states, trans = b.lkv_gdn_chunk_artifacts(k, v, g, beta, cu_seqlens=cu, compute=compute)
+    _, states2 = b.lkv_gdn_fwd(k, k, v, g, beta, cu_seqlens=cu, want_outputs=False, compute=compute)
+    trans2 = b.lkv_gdn_chunk_transition(k, g, beta, cu_seqlens=cu, compute=compute)
+    assert torch.equal(states, states2) and torch.equal(trans, trans2)
+    assert float(states[2].abs().max()) == 0.0 and torch.equal(trans[2, 0], torch.eye(128, device="cuda"))   # the empty chunk
