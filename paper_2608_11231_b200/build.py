@@ -30,10 +30,13 @@ def build(verbose: bool = False, force: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
     objs, procs = [], []
-    for src in sorted(glob.glob(os.path.join(CSRC, "*.cu"))):
+    sources = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+    # one stale source means a full rebuild (a few seconds): the library is never a mix of objects from different states
+    force = force or any(_newer(src, os.path.join(OBJ, os.path.basename(src)[:-3] + ".o"), headers) for src in sources)
+    for src in sources:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        if force or _newer(src, obj, headers):
+        if force:
             log = open(obj + ".log", "w")
             procs.append((src, log, subprocess.Popen([nvcc, *NVCC_FLAGS, "-c", src, "-o", obj],
                                                      stdout=log, stderr=subprocess.STDOUT)))
