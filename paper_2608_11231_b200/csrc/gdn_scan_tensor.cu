@@ -349,6 +349,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             if (has_o) tma_prefetch_desc(&mapO);
 #pragma unroll 1
             for (int b = 0; b < nblk + 2; ++b) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 const int st = b & 1;
                 const int row = t_begin + b * kC;
                 if (has_v && b + 2 < nblk)
@@ -428,6 +429,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             tma_prefetch_desc(&mapK);
 #pragma unroll 1
             for (int b = 0; b < nblk; ++b) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 const int s3 = b % kQKStages;
                 const int row = t_begin + b * kC;
                 unsigned char *base = sm + s3 * kQKStage;
@@ -911,6 +913,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             mbar_arrive(&bars.chain_done[b & 3]);
         }
     }
+    grace_after_timeout(&dead);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 17) tmem_dealloc(tm, kTmemCols);

@@ -108,6 +108,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
             };
             for (int j = 1; j < K && j <= kStages; ++j) load_T(j);
             for (int j = 1; j + kStages < K; ++j) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 // T_{j+kStages} takes over the stage of T_j as soon as the MMAs of step j are done
                 mbar_wait(&bar_freeT[stage_of(j)], phase_of(j), &dead, a.status);
                 load_T(j + kStages);
@@ -119,6 +120,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
             constexpr uint32_t idesc = umma_idesc(kFmtTF32, false, false, kD, 64);
             const uint64_t desc_hi = umma_desc(0, 0, 1024) & 0xFFFFFFFF00000000ull;
             for (int j = 1; j < K; ++j) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 const uint32_t lo0 = (smem_u32(sm + stage_of(j) * kTStageBytes) & 0x3FFFFu) >> 4;
                 const uint32_t abuf = tacc + 256 + 128 * ((j - 1) & 1);
                 const uint32_t dbuf = tacc + 128 * (j & 1);
@@ -222,6 +224,7 @@ init_gdn_exact_tensor_kernel(const __grid_constant__ InitArgs a, const __grid_co
             }
         }
     }
+    grace_after_timeout(&dead);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == kMmaWarp) tmem_dealloc(tacc, kTmemCols);

@@ -85,6 +85,7 @@ init_mamba_exact_stream_kernel(const __grid_constant__ InitArgs a, size_t state_
                 __syncwarp();
                 if (lane == 0) {
                     for (int jj = 0; jj < nj; ++jj, ++it) {
+                        if (dead) break;   // a wait ran out: nothing more is issued
                         const int s = it % kStages;
                         if (it >= kStages) mbar_wait(&empty[s], ((it / kStages) & 1) ^ 1, &dead, a.status);
                         const size_t c = static_cast<size_t>(a.id(k0 + j0 + jj));
@@ -156,6 +157,7 @@ init_mamba_exact_stream_kernel(const __grid_constant__ InitArgs a, size_t state_
                                make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]));
         }
     }
+    grace_after_timeout(&dead);   // copies still in flight land before the ring is given back
 }
 
 }  // namespace

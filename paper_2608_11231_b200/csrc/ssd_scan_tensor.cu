@@ -121,6 +121,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             tma_prefetch_desc(&mapC);
             if (a.y) tma_prefetch_desc(&mapY);
             for (int b = 0; b < nblk + 2; ++b) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 const int st = b & 1;
                 unsigned char *base = sm + st * kStageBytes;
                 const int row = t_begin + b * kQ;
@@ -180,6 +181,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             tc_fence_after_sync();
             issue_a(0);
             for (int b = 0; b < nblk; ++b) {
+                if (dead) break;   // a wait ran out: nothing more is issued
                 const uint32_t par = b & 1;
                 const uint32_t sbase_u = smem_u32(sm + (b & 1) * kStageBytes);
                 const uint64_t dX = umma_desc(sbase_u, 0, 1024);
@@ -475,6 +477,7 @@ ssd_scan_tensor_kernel(const __grid_constant__ SsdArgs a, const __grid_constant_
             mbar_arrive(&bars.yo_done[b % 3]);
         }
     }
+    grace_after_timeout(&dead);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 17) tmem_dealloc(tm, kTmemCols);

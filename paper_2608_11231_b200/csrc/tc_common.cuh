@@ -85,6 +85,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return mbar_wait_slow(smem_u32(bar), parity, dead, status, limit);
 }
 
+// After a wait has run out the threads that issue tile loads stop issuing (they test the flag once per block; an MMA
+// issuer may run through its remaining blocks without waiting, its products read whatever the tiles hold).  This pause,
+// taken by every thread before shared and tensor memory are given back, lets the loads and MMAs that were already in
+// flight land first.  They complete within a few microseconds; the pause is 64.
+__device__ __forceinline__ void grace_after_timeout(volatile int *dead) {
+    if (*dead)
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+}
+
 // ------------------------------------------------------------------ TMA (tiled bulk tensor loads, 2-D)
 // The innermost coordinate x times the element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
