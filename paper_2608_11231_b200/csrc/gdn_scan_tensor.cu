@@ -731,19 +731,20 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll
                         for (int c = 0; c < 16; c += 4) {
                             const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                            v[c] = __uint_as_float(rr[c]) * aa * f.x;
-                            v[c + 1] = __uint_as_float(rr[c + 1]) * aa * f.y;
-                            v[c + 2] = __uint_as_float(rr[c + 2]) * aa * f.z;
-                            v[c + 3] = __uint_as_float(rr[c + 3]) * aa * f.w;
+                            const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(rr[c]), __uint_as_float(rr[c + 1])), __fmul2_rn(make_float2(aa, aa), make_float2(f.x, f.y)));
+                            const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(rr[c + 2]), __uint_as_float(rr[c + 3])), __fmul2_rn(make_float2(aa, aa), make_float2(f.z, f.w)));
+                            v[c] = p0.x; v[c + 1] = p0.y; v[c + 2] = p1.x; v[c + 3] = p1.y;
                         }
                     } else {
 #pragma unroll
                         for (int c = 0; c < 16; c += 4) {
                             const float4 f = *reinterpret_cast<const float4 *>(sc + 4 * kC + i0 + c);
-                            v[c] = (i0 + c <= lim) ? __uint_as_float(rr[c]) * aa * f.x : 0.f;
-                            v[c + 1] = (i0 + c + 1 <= lim) ? __uint_as_float(rr[c + 1]) * aa * f.y : 0.f;
-                            v[c + 2] = (i0 + c + 2 <= lim) ? __uint_as_float(rr[c + 2]) * aa * f.z : 0.f;
-                            v[c + 3] = (i0 + c + 3 <= lim) ? __uint_as_float(rr[c + 3]) * aa * f.w : 0.f;
+                            const float2 p0 = __fmul2_rn(make_float2(__uint_as_float(rr[c]), __uint_as_float(rr[c + 1])), __fmul2_rn(make_float2(aa, aa), make_float2(f.x, f.y)));
+                            const float2 p1 = __fmul2_rn(make_float2(__uint_as_float(rr[c + 2]), __uint_as_float(rr[c + 3])), __fmul2_rn(make_float2(aa, aa), make_float2(f.z, f.w)));
+                            v[c] = (i0 + c <= lim) ? p0.x : 0.f;
+                            v[c + 1] = (i0 + c + 1 <= lim) ? p0.y : 0.f;
+                            v[c + 2] = (i0 + c + 2 <= lim) ? p1.x : 0.f;
+                            v[c + 3] = (i0 + c + 3 <= lim) ? p1.y : 0.f;
                         }
                     }
                     if (x < kC) {
@@ -808,10 +809,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 16; c += 4) {
                         const float4 ga = *reinterpret_cast<const float4 *>(sc + 2 * kC + 32 * half + 16 * q + c);
-                        v[c] = -ga.x * __uint_as_float(rr[q][c]);
-                        v[c + 1] = -ga.y * __uint_as_float(rr[q][c + 1]);
-                        v[c + 2] = -ga.z * __uint_as_float(rr[q][c + 2]);
-                        v[c + 3] = -ga.w * __uint_as_float(rr[q][c + 3]);
+                        const float2 p0 = __fmul2_rn(make_float2(-ga.x, -ga.y), make_float2(__uint_as_float(rr[q][c]), __uint_as_float(rr[q][c + 1])));
+                        const float2 p1 = __fmul2_rn(make_float2(-ga.z, -ga.w), make_float2(__uint_as_float(rr[q][c + 2]), __uint_as_float(rr[q][c + 3])));
+                        v[c] = p0.x; v[c + 1] = p0.y; v[c + 2] = p1.x; v[c + 3] = p1.y;
                     }
                     pack16(v, w[q]);
                 }
@@ -844,10 +844,9 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 16; c += 4) {
                         const float4 w4 = *reinterpret_cast<const float4 *>(sc + 3 * kC + 32 * half + 16 * q + c);
-                        v[c] = w4.x * __uint_as_float(rr[q][c]);
-                        v[c + 1] = w4.y * __uint_as_float(rr[q][c + 1]);
-                        v[c + 2] = w4.z * __uint_as_float(rr[q][c + 2]);
-                        v[c + 3] = w4.w * __uint_as_float(rr[q][c + 3]);
+                        const float2 p0 = __fmul2_rn(make_float2(w4.x, w4.y), make_float2(__uint_as_float(rr[q][c]), __uint_as_float(rr[q][c + 1])));
+                        const float2 p1 = __fmul2_rn(make_float2(w4.z, w4.w), make_float2(__uint_as_float(rr[q][c + 2]), __uint_as_float(rr[q][c + 3])));
+                        v[c] = p0.x; v[c + 1] = p0.y; v[c + 2] = p1.x; v[c + 3] = p1.y;
                     }
                     pack16(v, w[q]);
 #pragma unroll
@@ -903,7 +902,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) rr[q][c] = __float_as_uint(__uint_as_float(rr[q][c]) * gamN);
+                    for (int c = 0; c < 16; c += 2) {
+                        const float2 p = __fmul2_rn(make_float2(gamN, gamN), make_float2(__uint_as_float(rr[q][c]), __uint_as_float(rr[q][c + 1])));
+                        rr[q][c] = __float_as_uint(p.x);
+                        rr[q][c + 1] = __float_as_uint(p.y);
+                    }
                     tmem_st16(lane_base + kTmS + 64 * half + 16 * q, rr[q]);
                 }
                 tmem_st_wait();
