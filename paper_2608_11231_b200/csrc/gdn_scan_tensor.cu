@@ -359,7 +359,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 if (b >= 2) {
                     mbar_wait(&bars.o_staged[st], ((b - 2) >> 1) & 1, &dead, a.status);
                     if (has_o && row - kC <= t_end && !dead) {
-                        tma_store_2d(&mapO, sm + kOffV + st * kVStage, h * kD, row - 2 * kC);
+                        for (int jb = 0; jb < 2; ++jb) tma_store_2d(&mapO, sm + kOffV + st * kVStage + jb * kC * 128, h * kD + jb * 64, row - 2 * kC);
                         tma_store_commit();
                         tma_store_wait_read();
                     }
@@ -663,21 +663,34 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             const int t0 = t_begin + b * kC;
             const int n = min(kC, t_end - t0);
             if (has_o && (n == kC || !dead)) {
-                // whole block: stage the tile in the V stage of this block, which (3a) has finished reading; the
-                // store warp writes it out with TMA
-                __nv_bfloat16 *os = reinterpret_cast<__nv_bfloat16 *>(sm + kOffV + (b & 1) * kVStage) + x;
+                if (n != kC) {
+                    // ragged last block: straight to global memory, 16 tokens of one state column per call
 #pragma unroll 1
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t taddr = lane_base + kTmO + 64 * (b & 1) + 16 * q;
-                    if (n != kC) {
-                        store_o_partial(taddr, o + (static_cast<size_t>(t0 + 16 * q) * a.H_v + h) * kD + x, tstride, n - 16 * q);
-                        continue;
-                    }
-                    uint32_t pu[16];
-                    tmem_ld16(taddr, pu);
-                    tmem_ld_wait();
+                    for (int q = 0; q < 4; ++q)
+                        store_o_partial(lane_base + kTmO + 64 * (b & 1) + 16 * q, o + (static_cast<size_t>(t0 + 16 * q) * a.H_v + h) * kD + x,
+                                        tstride, n - 16 * q);
+                } else {
+                    // whole block: stage the tile in the V stage of this block, which (3a) has finished reading, in the layout of
+                    // the tensor map (two halves of 64 features, 128-byte rows, 128-byte swizzle); the store warp writes it out
+                    // with TMA.  O^T leaves tensor memory in accumulator layout (thread = feature, register pair = two tokens) and
+                    // is stored transposed, 16 features x 16 tokens per instruction.
+                    unsigned char *os = sm + kOffV + (b & 1) * kVStage + (warp & 2 ? kC * 128 : 0);
+                    const int m = lane >> 3, i = lane & 7;
+#pragma unroll 1
+                    for (int lh = 0; lh < 2; ++lh) {
+                        uint32_t pu[32];
+                        tmem_ld_16x256b_x8(lane_base + (static_cast<uint32_t>(16 * lh) << 16) + kTmO + 64 * (b & 1), pu);
+                        tmem_ld_wait();
+                        const int chunk = 4 * (warp & 1) + 2 * lh + (m & 1);   // 16-byte piece of the 128-byte row: 8 features
+                        const uint32_t row_addr = smem_u32(os) + (8 * (m >> 1) + i) * 128 + ((chunk ^ i) << 4);
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) os[(16 * q + c) * kD] = __float2bfloat16_rn(__uint_as_float(pu[c]));
+                        for (int kk = 0; kk < 4; ++kk)   // tokens 16 kk .. 16 kk + 15
+                            stmatrix_x4_trans(row_addr + 16 * kk * 128,
+                                              pack_bf16(__uint_as_float(pu[8 * kk]), __uint_as_float(pu[8 * kk + 1])),
+                                              pack_bf16(__uint_as_float(pu[8 * kk + 2]), __uint_as_float(pu[8 * kk + 3])),
+                                              pack_bf16(__uint_as_float(pu[8 * kk + 4]), __uint_as_float(pu[8 * kk + 5])),
+                                              pack_bf16(__uint_as_float(pu[8 * kk + 6]), __uint_as_float(pu[8 * kk + 7])));
+                    }
                 }
                 fence_async_smem();
             }
@@ -940,7 +953,7 @@ cudaError_t launch_gdn_scan_tensor(const GdnArgs &a, cudaStream_t s) {
     } else if (!make_tensor_map_2d(&mapQ, a.q, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         !make_tensor_map_2d(&mapK, a.k, 2, qk_inner, rows, qk_inner * 2, 64, kC, true) ||
         (a.v && !make_tensor_map_2d(&mapV, a.v, 2, v_inner, rows, v_inner * 2, 64, kC, true)) ||
-        (a.o && !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, kD, kC, false)))
+        (a.o && !make_tensor_map_2d(&mapO, a.o, 2, v_inner, rows, v_inner * 2, 64, kC, true)))
         return cudaErrorInvalidValue;
     if (!a.v) mapV = mapK;   // never used by the kernel then
     if (!a.o) mapO = mapK;
