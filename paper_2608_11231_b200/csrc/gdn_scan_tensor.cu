@@ -553,10 +553,11 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
             unsigned char *xb = sm + kOffX + (b & 1) * (kC * 128);
             named_bar_sync(1, 128);   // every thread is done with the fp32 M of the previous block
             const float *Af = reinterpret_cast<const float *>(sm + kOffA) + (b & 1) * (kC * kLd);
-            // ---- M = (I + A)^{-1} by doubling.  8x8 diagonal blocks: thread (k, c) solves column c of block k by forward
-            // substitution (fp32).
-            if (x < kC) {
-                const int k = x >> 3, c = x & 7;
+            // ---- M = (I + A)^{-1} by doubling.  Warp w owns the 16x16 diagonal block w up to the 8 -> 16 merge, so that the two
+            // steps need no barrier between the warps.  8x8 diagonal blocks 2w, 2w+1: lane (kk, c) solves column c of block
+            // 2w + kk by forward substitution (fp32).
+            if (lane < 16) {
+                const int k = 2 * (warp & 3) + (lane >> 3), c = lane & 7;
                 const float *Ab = Af + (8 * k) * kLd + 8 * k;
                 float xv[8];
 #pragma unroll
@@ -584,8 +585,8 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 for (int t = 0; t < 8; ++t)
                     *reinterpret_cast<__nv_bfloat16 *>(xb + x_offset(8 * k + t, 8 * k + c)) = __float2bfloat16_rn(xv[t] * bc);
             }
-            named_bar_sync(1, 128);
-            // 8 -> 16 in fp32: thread = (16-block k, row i, column pair) of the 8x8 block below the diagonal;
+            __syncwarp();
+            // 8 -> 16 in fp32: thread = (16-block k = this warp, row i, column pair) of the 8x8 block below the diagonal;
             // T = A21 inv(L1) passes through the scratch M[0..31, 32..39]
             {
                 const int k = x >> 5, i = (x >> 2) & 7, j0 = 2 * (x & 3);
@@ -600,7 +601,7 @@ gdn_scan_tensor_kernel(const __grid_constant__ GdnArgs a, const __grid_constant_
                 }
                 float *ts = Mf + (8 * k) * kLd + 32;
                 *reinterpret_cast<float2 *>(ts + i * kLd + j0) = make_float2(t0, t1);
-                named_bar_sync(1, 128);
+                __syncwarp();
                 const float *d2 = Mf + (16 * k + 8 + i) * kLd + 16 * k + 8;
                 float m0 = 0.f, m1 = 0.f;
 #pragma unroll
