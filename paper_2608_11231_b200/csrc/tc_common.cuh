@@ -78,10 +78,12 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
     if (status) atomicExch(status, 1);
     return false;
 }
-// The probe is inline (the common case in a pipeline that runs ahead); the polling loop is one shared
-// function so that the many waits of a warp-specialised kernel do not bloat its instruction footprint.
+// The first probe is inline and is a try_wait: it returns at once when the phase is complete and otherwise suspends the
+// thread until it completes or a window of several thousand cycles has passed, so a wait of ordinary length costs this
+// one instruction.  Only a wait that outlasts the window enters the polling loop, which is one shared function so that
+// the many waits of a warp-specialised kernel do not bloat its instruction footprint.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status, uint32_t limit = kSpinLimit) {
-    if (mbar_test_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(smem_u32(bar), parity, dead, status, limit);
 }
 
