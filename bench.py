@@ -63,7 +63,7 @@ def ssd_scan_flops(tokens: int, s=SSD_SHAPE, Q=SSD_BLOCK) -> float:
 # DRAM bytes (read + write) per scanned token from ncu captures of one launch of each scan kernel (GDN: 8 sequences x
 # 2048 tokens; Mamba-2: 16 sequences x 4096 tokens, initial and final states included); the traffic of a scan grows
 # in proportion to its tokens.
-NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.47e6 + 119.68e6) / 16384, "mamba2.scan": (788.94e6 + 671.04e6) / 65536}
+NCU_DRAM_BYTES_PER_TOKEN = {"gdn.scan": (290.48e6 + 119.29e6) / 16384, "mamba2.scan": (789.18e6 + 672.45e6) / 65536}
 
 
 def gdn_scan_bytes(tokens: int, s=GDN_SHAPE) -> float:
