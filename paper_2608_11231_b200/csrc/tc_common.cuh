@@ -20,7 +20,8 @@ __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.f
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // ------------------------------------------------------------------ mbarriers (all waits bounded)
-constexpr uint32_t kSpinLimit = 1u << 22;  // try_wait polls before a wait gives up (each poll suspends the thread briefly)
+constexpr uint32_t kSpinLimit = 1u << 18;  // try_wait polls before a wait gives up: a poll that fails has suspended the thread for about
+                                           // 7.8 K cycles, so this is about a second; no wait of a working pipeline comes near it
 
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
